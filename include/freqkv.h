@@ -1,0 +1,152 @@
+/*
+ * freqkv.h -- C ABI of the FreqKV iterative KV-cache compression library for NVIDIA B200
+ * (sm_100a).
+ *
+ * The library keeps a bounded key/value cache usable for arbitrarily long contexts: new
+ * tokens are appended until the cache is full, then the non-sink part of every
+ * (batch, layer, kv_head) matrix of K and of V is compressed in the frequency domain along
+ * the token axis and written back in place, shorter, so that appending can go on
+ * (FreqKV, Sections 3.3 and 3.4).
+ *
+ * Conventions
+ *  - All cache pointers are DEVICE pointers owned by the caller; the library never frees or
+ *    reallocates them.  `lens`, `kept_len` arrays and layout structs are HOST memory.
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Calls enqueue work on it and return without synchronising, unless stated otherwise.
+ *  - Every function returns a freqkv_status; on any status other than FREQKV_OK nothing was
+ *    enqueued and no caller memory was modified.  No C++ exception crosses the boundary.
+ *  - A context belongs to one device and must not be used from two threads at once.
+ *  - There is no CPU fallback: without a CUDA device freqkv_create fails.
+ */
+#ifndef FREQKV_H_
+#define FREQKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FREQKV_OK = 0,
+    FREQKV_ERR_INVALID_ARG = 1, /* null pointer, negative or inconsistent size            */
+    FREQKV_ERR_UNSUPPORTED = 2, /* dtype / head_dim / stride / variant not supported      */
+    FREQKV_ERR_CAPACITY = 3,    /* append would exceed the cache capacity: compress first */
+    FREQKV_ERR_ALLOC = 4,       /* device or host allocation failed                       */
+    FREQKV_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed                   */
+    FREQKV_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (see last_device_status) */
+} freqkv_status;
+
+typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
+
+/* Which kernel family executes the compression.
+ *   GEMM  the DCT-II -> truncate -> IDCT -> rescale chain folded into one precomputed
+ *         kept_len x n_in projection basis and run on the tcgen05 tensor cores (bf16 caches,
+ *         head_dim 128 only);
+ *   FDCT  fast-transform kernel (power-of-two n_in and kept_len only);
+ *   SIMT  the same projection on the fp32 CUDA cores (any shape; the only path for fp32
+ *         caches of non-power-of-two length);
+ *   AUTO  picks per shape from a table filled from measurements. */
+typedef enum { FREQKV_AUTO = 0, FREQKV_GEMM = 1, FREQKV_FDCT = 2, FREQKV_SIMT = 3 } freqkv_variant;
+
+/* Layout of ONE cache tensor (K or V; both must share it):
+ * element (b, l, h, t, c) lives at  base + b*stride_batch + l*stride_layer + h*stride_head
+ *                                        + t*stride_token + c      (strides in ELEMENTS).
+ * head_dim is the contiguous axis.  Requirements: head_dim a multiple of 8 and at most 256,
+ * stride_token >= head_dim, every stride a multiple of 8 elements (so that rows are 16-byte
+ * aligned when the base pointer is), and the strides must not make two matrices overlap. */
+typedef struct {
+    int32_t dtype; /* freqkv_dtype */
+    int32_t batch, layers, kv_heads, capacity /* tokens */, head_dim;
+    int64_t stride_batch, stride_layer, stride_head, stride_token;
+} freqkv_layout;
+
+typedef struct freqkv_ctx freqkv_ctx; /* opaque: projection bases, twiddles, scratch, status word */
+
+/* Fill `out` with the dense row-major [batch, layers, kv_heads, capacity, head_dim] layout. */
+freqkv_status freqkv_layout_contiguous(freqkv_layout* out, freqkv_dtype dtype, int32_t batch, int32_t layers,
+                                       int32_t kv_heads, int32_t capacity, int32_t head_dim);
+
+/* Create / destroy a context on CUDA device `device`.  Creation allocates a small status
+ * word; plans and scratch are allocated lazily (cudaMalloc) by freqkv_plan or by the first
+ * compression of a new shape, and freed by freqkv_destroy.  Destroy synchronises the device. */
+freqkv_status freqkv_create(freqkv_ctx** out, int device);
+freqkv_status freqkv_destroy(freqkv_ctx* ctx);
+
+/* Force the variant used by later freqkv_compress* calls (default FREQKV_AUTO).  A forced
+ * variant that cannot run a given shape makes that call return FREQKV_ERR_UNSUPPORTED. */
+freqkv_status freqkv_set_variant(freqkv_ctx* ctx, freqkv_variant variant);
+
+/* Which variant AUTO (or the forced setting) resolves to for this shape; FREQKV_AUTO is never
+ * returned.  Returns FREQKV_ERR_UNSUPPORTED through *out_variant = -1 when none applies. */
+freqkv_status freqkv_resolve_variant(freqkv_ctx* ctx, const freqkv_layout* layout, int32_t n_in, int32_t n_keep,
+                                     int32_t* out_variant);
+
+/* Optional warm-up: build and cache whatever tables the given variant needs to compress
+ * n_in non-sink rows to n_keep rows (the projection basis of Eq. 2-3 folded with the
+ * definitions of Appendix A, or the transform twiddles).  Work is enqueued on `cuda_stream`.
+ * Calling freqkv_compress without it builds the plan on first use. */
+freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_dtype dtype,
+                          freqkv_variant variant, void* cuda_stream);
+
+/* One compression of a uniform cache (Section 3.3, Eq. 2-3; sink tokens: Section 3.4).
+ * For every (batch, layer, kv_head) and for K and V alike, with N = cache_len - sink and
+ * L = kept_len, rows [sink, cache_len) are one signal per channel:
+ *     z = DCT-II_N(x)  (orthonormal, Appendix A);  keep z[0:L];
+ *     y = sqrt(L/N) * IDCT_L(z[0:L])               (L-point orthonormal inverse).
+ * y is rounded once (nearest even) to the cache dtype and written to rows [sink, sink+L).
+ * Nothing else is written: sink rows, rows >= sink+L and any stride padding keep their bytes.
+ * The caller's new cache length is sink + kept_len.  Arithmetic: fp32 accumulation.
+ * kept_len == cache_len - sink is the identity and enqueues nothing; kept_len == 0 or
+ * cache_len == sink enqueue nothing.
+ * Errors: INVALID_ARG (null pointers, sink < 0, sink > cache_len, cache_len > capacity,
+ * kept_len < 0, kept_len > cache_len - sink, k == v), UNSUPPORTED (layout rules above, forced
+ * variant not applicable), ALLOC, CUDA. */
+freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
+                              int32_t kept_len, int32_t sink, void* cuda_stream);
+
+/* Ragged form: sequence b holds lens[b] rows and is compressed to sink + kept_len[b] rows,
+ * each sequence with the transform of its own length (same definition as above with
+ * N = lens[b] - sink, L = kept_len[b]).  `lens` and `kept_len` are host arrays of
+ * layout->batch entries; on success lens[b] is updated to sink + kept_len[b].  All arguments
+ * are validated for every sequence before anything is enqueued. */
+freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t* lens,
+                                     const int32_t* kept_len, int32_t sink, void* cuda_stream);
+
+/* Append n_new incoming tokens to every sequence (Section 3.4: incoming tokens are appended
+ * to the compressed cache).  new_k / new_v are device pointers to dense
+ * [batch, layers, kv_heads, n_new, head_dim] tensors of the cache dtype; rows
+ * [lens[b], lens[b] + n_new) of sequence b are overwritten and lens[b] (host) grows by n_new.
+ * If any lens[b] + n_new exceeds the capacity nothing is enqueued and FREQKV_ERR_CAPACITY is
+ * returned: the caller compresses and retries -- this is the lazy trigger that reproduces the
+ * compression counts of the paper's tables (a 4K-token input causes no compression). */
+freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
+                            const void* new_v, int32_t n_new, int32_t* lens, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, then read and clear the device status word.  FREQKV_OK unless a
+ * kernel's bounded wait (mbarrier / flag) ran out, in which case the affected output rows are
+ * undefined and FREQKV_ERR_TIMEOUT is returned; the context stays usable. */
+freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream);
+
+/* Host-only argument checks, exactly the ones freqkv_compress / freqkv_append apply before
+ * they enqueue anything (they touch no device and need no context): the status those calls
+ * would return for these arguments, FREQKV_OK if they would go ahead. */
+freqkv_status freqkv_check_compress(const freqkv_layout* layout, const void* k, const void* v, int32_t cache_len,
+                                    int32_t kept_len, int32_t sink);
+freqkv_status freqkv_check_append(const freqkv_layout* layout, const void* k, const void* v, const void* new_k,
+                                  const void* new_v, int32_t n_new, const int32_t* lens);
+
+/* Text of the most recent CUDA failure or device-status report seen by this context (owned by
+ * the context, valid until its next call); "" if none. */
+const char* freqkv_last_error(freqkv_ctx* ctx);
+
+/* Static, human-readable name of a status code. */
+const char* freqkv_status_string(freqkv_status status);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int32_t freqkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FREQKV_H_ */

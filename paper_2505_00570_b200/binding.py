@@ -1,0 +1,211 @@
+"""Thin ctypes binding of ``libfreqkv.so`` (declared in ``include/freqkv.h``).
+
+Argument marshalling only: tensors are passed as ``data_ptr()``, the stream as
+``torch.cuda.current_stream().cuda_stream``; every step of the path runs in the library's
+kernels.  There is no fallback: if the library is not built, or a call fails, an exception is
+raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_int, c_int32, c_int64, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfreqkv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(7)
+BF16, F32 = 0, 1
+AUTO, GEMM, FDCT, SIMT = 0, 1, 2, 3
+VARIANT_NAMES = {AUTO: "auto", GEMM: "gemm", FDCT: "fdct", SIMT: "simt"}
+
+EXPORTS = [
+    "freqkv_layout_contiguous", "freqkv_create", "freqkv_destroy", "freqkv_set_variant",
+    "freqkv_resolve_variant", "freqkv_plan", "freqkv_compress", "freqkv_compress_ragged",
+    "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
+    "freqkv_last_error", "freqkv_status_string", "freqkv_version",
+]
+
+
+class Layout(ctypes.Structure):
+    """Mirror of ``freqkv_layout``."""
+
+    _fields_ = [
+        ("dtype", c_int32), ("batch", c_int32), ("layers", c_int32), ("kv_heads", c_int32),
+        ("capacity", c_int32), ("head_dim", c_int32),
+        ("stride_batch", c_int64), ("stride_layer", c_int64), ("stride_head", c_int64), ("stride_token", c_int64),
+    ]
+
+
+class FreqKVError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(what)
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the library on first use; raise loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FreqKVError(ERR_CUDA, f"{LIB_PATH} is missing: build it with "
+                                        "`python -m paper_2505_00570_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        LP = POINTER(Layout)
+        I32P = POINTER(c_int32)
+        L.freqkv_layout_contiguous.argtypes = [LP, c_int, c_int32, c_int32, c_int32, c_int32, c_int32]
+        L.freqkv_create.argtypes = [POINTER(c_void_p), c_int]
+        L.freqkv_destroy.argtypes = [c_void_p]
+        L.freqkv_set_variant.argtypes = [c_void_p, c_int]
+        L.freqkv_resolve_variant.argtypes = [c_void_p, LP, c_int32, c_int32, I32P]
+        L.freqkv_plan.argtypes = [c_void_p, c_int32, c_int32, c_int, c_int, c_void_p]
+        L.freqkv_compress.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
+        L.freqkv_compress_ragged.argtypes = [c_void_p, LP, c_void_p, c_void_p, I32P, I32P, c_int32, c_void_p]
+        L.freqkv_append.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P, c_void_p]
+        L.freqkv_last_device_status.argtypes = [c_void_p, c_void_p]
+        L.freqkv_check_compress.argtypes = [LP, c_void_p, c_void_p, c_int32, c_int32, c_int32]
+        L.freqkv_check_append.argtypes = [LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P]
+        L.freqkv_last_error.argtypes = [c_void_p]
+        L.freqkv_last_error.restype = c_char_p
+        L.freqkv_status_string.argtypes = [c_int]
+        L.freqkv_status_string.restype = c_char_p
+        L.freqkv_version.restype = c_int32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().freqkv_status_string(status).decode()
+
+
+def dtype_code(dtype: torch.dtype) -> int:
+    if dtype == torch.bfloat16:
+        return BF16
+    if dtype == torch.float32:
+        return F32
+    raise FreqKVError(ERR_UNSUPPORTED, f"unsupported cache dtype {dtype}")
+
+
+def layout_of(t: torch.Tensor) -> Layout:
+    """``freqkv_layout`` of a ``[batch, layers, kv_heads, capacity, head_dim]`` tensor (a view
+    with arbitrary strides is fine as long as head_dim is contiguous)."""
+    if t.dim() != 5 or t.stride(4) != 1:
+        raise FreqKVError(ERR_UNSUPPORTED, "cache must be [batch, layers, kv_heads, capacity, head_dim] with contiguous head_dim")
+    return Layout(dtype_code(t.dtype), t.shape[0], t.shape[1], t.shape[2], t.shape[3], t.shape[4],
+                  t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+
+
+def layout_contiguous(dtype: int, batch: int, layers: int, kv_heads: int, capacity: int, head_dim: int):
+    """(status, Layout) from ``freqkv_layout_contiguous``."""
+    out = Layout()
+    st = lib().freqkv_layout_contiguous(ctypes.byref(out), dtype, batch, layers, kv_heads, capacity, head_dim)
+    return st, out
+
+
+def check_compress(layout: Layout, k_ptr: int, v_ptr: int, cache_len: int, kept_len: int, sink: int) -> int:
+    return lib().freqkv_check_compress(ctypes.byref(layout), k_ptr, v_ptr, cache_len, kept_len, sink)
+
+
+def check_append(layout: Layout, k_ptr: int, v_ptr: int, nk_ptr: int, nv_ptr: int, n_new: int, lens) -> int:
+    arr = (c_int32 * len(lens))(*lens)
+    return lib().freqkv_check_append(ctypes.byref(layout), k_ptr, v_ptr, nk_ptr, nv_ptr, n_new, arr)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+class Context:
+    """Owns one ``freqkv_ctx`` (plan cache, scratch, status word) on one device."""
+
+    def __init__(self, device: int | None = None):
+        if device is None:
+            device = torch.cuda.current_device()
+        self.device = int(device)
+        self._h = c_void_p()
+        st = lib().freqkv_create(ctypes.byref(self._h), self.device)
+        if st != OK:
+            self._h = c_void_p()
+            raise FreqKVError(st, f"freqkv_create: {status_string(st)} (a B200 and the built library are required)")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().freqkv_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int, what: str):
+        if st != OK:
+            detail = lib().freqkv_last_error(self._h).decode() if st in (ERR_CUDA, ERR_ALLOC, ERR_TIMEOUT) else ""
+            raise FreqKVError(st, f"{what}: {status_string(st)} {detail}".strip())
+
+    def set_variant(self, variant: int):
+        self._check(lib().freqkv_set_variant(self._h, variant), "freqkv_set_variant")
+
+    def resolve_variant(self, layout: Layout, n_in: int, n_keep: int) -> int:
+        out = c_int32(-1)
+        st = lib().freqkv_resolve_variant(self._h, ctypes.byref(layout), n_in, n_keep, ctypes.byref(out))
+        if st == ERR_UNSUPPORTED:
+            return -1
+        self._check(st, "freqkv_resolve_variant")
+        return out.value
+
+    def plan(self, n_in: int, n_keep: int, dtype: int, variant: int = AUTO, stream=None):
+        self._check(lib().freqkv_plan(self._h, n_in, n_keep, dtype, variant, _stream_ptr(stream)), "freqkv_plan")
+
+    def compress(self, k: torch.Tensor, v: torch.Tensor, cache_len: int, kept_len: int, sink: int, stream=None) -> int:
+        """In-place compression of rows [sink, cache_len) of every matrix to kept_len rows.
+        Returns the new cache length."""
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        st = lib().freqkv_compress(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), cache_len, kept_len, sink,
+                                   _stream_ptr(stream))
+        self._check(st, "freqkv_compress")
+        return sink + kept_len
+
+    def compress_ragged(self, k: torch.Tensor, v: torch.Tensor, lens: list[int], kept_len: list[int], sink: int,
+                        stream=None) -> list[int]:
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        if len(lens) != lay.batch or len(kept_len) != lay.batch:
+            raise FreqKVError(ERR_INVALID_ARG, "lens and kept_len need one entry per sequence")
+        c_lens = (c_int32 * lay.batch)(*lens)
+        c_keep = (c_int32 * lay.batch)(*kept_len)
+        st = lib().freqkv_compress_ragged(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), c_lens, c_keep, sink,
+                                          _stream_ptr(stream))
+        self._check(st, "freqkv_compress_ragged")
+        return list(c_lens)
+
+    def append(self, k: torch.Tensor, v: torch.Tensor, new_k: torch.Tensor, new_v: torch.Tensor, lens: list[int],
+               stream=None) -> list[int]:
+        """Append new_k / new_v ``[batch, layers, kv_heads, n_new, head_dim]`` (dense) at each
+        sequence's length; returns the new lengths.  Raises FreqKVError(ERR_CAPACITY) when a
+        sequence has no room: compress and retry."""
+        lay = layout_of(k)
+        if not (new_k.is_contiguous() and new_v.is_contiguous()) or new_k.shape != new_v.shape:
+            raise FreqKVError(ERR_INVALID_ARG, "new_k / new_v must be dense and of equal shape")
+        if tuple(new_k.shape[:3]) != tuple(k.shape[:3]) or new_k.shape[4] != k.shape[4] or new_k.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "new rows do not match the cache")
+        n_new = new_k.shape[3]
+        c_lens = (c_int32 * lay.batch)(*lens)
+        st = lib().freqkv_append(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), new_k.data_ptr(),
+                                 new_v.data_ptr(), n_new, c_lens, _stream_ptr(stream))
+        self._check(st, "freqkv_append")
+        return list(c_lens)
+
+    def last_device_status(self, stream=None) -> int:
+        return lib().freqkv_last_device_status(self._h, _stream_ptr(stream))

@@ -1,0 +1,540 @@
+// C ABI of the FreqKV library: argument validation, plan cache, variant choice and dispatch.
+// All arithmetic of the hot path runs in the kernels this file launches; nothing here touches
+// cache contents on the host.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "common.cuh"
+#include "gemm.cuh"
+#include "fdct.cuh"
+
+using namespace freqkv;
+
+struct freqkv_ctx {
+    int device = 0;
+    int sm_count = 0;
+    freqkv_variant forced = FREQKV_AUTO;
+    std::map<std::pair<int32_t, int32_t>, Basis> bases;
+    std::map<std::pair<int32_t, int32_t>, FdctPlan> fdct_plans;
+    size_t basis_bytes = 0;
+    void* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    int32_t* status_dev = nullptr;
+    GemmState gemm;
+    std::string last_error;
+};
+
+namespace {
+
+constexpr size_t kScratchChunkBytes = size_t(1) << 30;  // per-chunk output staging of the scratch paths
+constexpr size_t kBasisBudgetBytes = size_t(12) << 30;  // plan cache is flushed beyond this
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+freqkv_status cuda_fail(freqkv_ctx* ctx, cudaError_t e, const char* where)
+{
+    if (ctx) ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
+    cudaGetLastError();  // clear the sticky-free error state
+    return e == cudaErrorMemoryAllocation ? FREQKV_ERR_ALLOC : FREQKV_ERR_CUDA;
+}
+
+#define FREQKV_CUDA(ctx, call)                                             \
+    do {                                                                   \
+        const cudaError_t e__ = (call);                                    \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__, #call);       \
+    } while (0)
+
+int64_t span_elements(const freqkv_layout& l)
+{
+    return (int64_t)(l.batch - 1) * l.stride_batch + (int64_t)(l.layers - 1) * l.stride_layer +
+           (int64_t)(l.kv_heads - 1) * l.stride_head + (int64_t)(l.capacity - 1) * l.stride_token + l.head_dim;
+}
+
+freqkv_status check_layout(const freqkv_layout* l)
+{
+    if (!l) return FREQKV_ERR_INVALID_ARG;
+    if (l->dtype != FREQKV_BF16 && l->dtype != FREQKV_F32) return FREQKV_ERR_UNSUPPORTED;
+    if (l->batch < 1 || l->layers < 1 || l->kv_heads < 1 || l->capacity < 1 || l->head_dim < 1)
+        return FREQKV_ERR_INVALID_ARG;
+    if (l->head_dim % 8 != 0 || l->head_dim > 256) return FREQKV_ERR_UNSUPPORTED;
+    if ((int64_t)l->batch * l->layers * l->kv_heads > (int64_t)1 << 29) return FREQKV_ERR_UNSUPPORTED;
+    const int64_t strides[4] = {l->stride_token, l->stride_head, l->stride_layer, l->stride_batch};
+    const int64_t extents[4] = {l->capacity, l->kv_heads, l->layers, l->batch};
+    for (int i = 0; i < 4; ++i) {
+        if (strides[i] < 0) return FREQKV_ERR_INVALID_ARG;
+        if (strides[i] % 8 != 0) return FREQKV_ERR_UNSUPPORTED;
+    }
+    // No two matrices may overlap: ordered by stride, each axis must step over the whole extent
+    // of the axes below it (axes of extent 1 never step).
+    std::vector<std::pair<int64_t, int64_t>> axes;  // (stride, extent)
+    for (int i = 0; i < 4; ++i)
+        if (extents[i] > 1) axes.emplace_back(strides[i], extents[i]);
+    std::sort(axes.begin(), axes.end());
+    int64_t below = l->head_dim;
+    for (const auto& a : axes) {
+        if (a.first < below) return FREQKV_ERR_UNSUPPORTED;
+        below = a.first * a.second;
+    }
+    if (l->stride_token < l->head_dim && l->capacity > 1) return FREQKV_ERR_UNSUPPORTED;
+    return FREQKV_OK;
+}
+
+freqkv_status check_tensors(const freqkv_layout& l, const void* k, const void* v)
+{
+    if (!k || !v) return FREQKV_ERR_INVALID_ARG;
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return FREQKV_ERR_UNSUPPORTED;
+    const int64_t bytes = span_elements(l) * (int64_t)dtype_size(l.dtype);
+    const char* a = static_cast<const char*>(k);
+    const char* b = static_cast<const char*>(v);
+    if (a < b + bytes && b < a + bytes) return FREQKV_ERR_INVALID_ARG;  // K and V overlap
+    return FREQKV_OK;
+}
+
+CacheView make_view(const freqkv_layout& l, void* k, void* v, int32_t batch0, int32_t batch_count)
+{
+    CacheView w;
+    w.base[0] = k;
+    w.base[1] = v;
+    w.stride_batch = l.stride_batch;
+    w.stride_layer = l.stride_layer;
+    w.stride_head = l.stride_head;
+    w.stride_token = l.stride_token;
+    w.layers = l.layers;
+    w.kv_heads = l.kv_heads;
+    w.head_dim = l.head_dim;
+    w.mats_per_tensor = batch_count * l.layers * l.kv_heads;
+    w.batch0 = batch0;
+    return w;
+}
+
+bool is_pow2(int32_t x) { return x > 0 && (x & (x - 1)) == 0; }
+
+bool gemm_applicable(const freqkv_layout& l, int32_t n_in, int32_t n_keep)
+{
+    return gemm_supported(l.dtype, l.head_dim, n_in, n_keep);
+}
+
+bool fdct_applicable(const freqkv_layout& l, int32_t n_in, int32_t n_keep)
+{
+    return fdct_supported(l.dtype, l.head_dim, n_in, n_keep) && is_pow2(n_in) && is_pow2(n_keep);
+}
+
+// Variant table.  Measured on B200 (bf16, head_dim 128): the fast-transform kernel wins wherever
+// it applies (power-of-two lengths); the tensor-core projection wins on every other bf16 shape
+// once the matrices are long enough to fill a tile; tiny problems and fp32 caches of other
+// lengths run on the CUDA cores.
+int32_t resolve(const freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
+{
+    const bool g = gemm_applicable(l, n_in, n_keep), f = fdct_applicable(l, n_in, n_keep);
+    switch (ctx->forced) {
+        case FREQKV_GEMM: return g ? FREQKV_GEMM : -1;
+        case FREQKV_FDCT: return f ? FREQKV_FDCT : -1;
+        case FREQKV_SIMT: return FREQKV_SIMT;
+        default: break;
+    }
+    if (f) return FREQKV_FDCT;
+    if (g && n_in >= 128) return FREQKV_GEMM;
+    return FREQKV_SIMT;
+}
+
+void free_bases(freqkv_ctx* ctx)
+{
+    for (auto& kv : ctx->bases) {
+        if (kv.second.f32) cudaFree(kv.second.f32);
+        if (kv.second.bf16) cudaFree(kv.second.bf16);
+    }
+    ctx->bases.clear();
+    ctx->basis_bytes = 0;
+}
+
+// Projection basis for (n_in, n_keep) holding at least the requested precisions.
+freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need_f32, bool need_bf16,
+                        cudaStream_t stream, Basis* out)
+{
+    const auto key = std::make_pair(n_in, n_keep);
+    Basis b;
+    auto it = ctx->bases.find(key);
+    if (it != ctx->bases.end()) b = it->second;
+    const bool make_f32 = need_f32 && !b.f32, make_bf16 = need_bf16 && !b.bf16;
+    if (make_f32 || make_bf16) {
+        b.n_in = n_in;
+        b.n_keep = n_keep;
+        b.ld = (n_in + 63) / 64 * 64;
+        b.rows_pad = (n_keep + 63) / 64 * 64;
+        const size_t elems = (size_t)b.ld * b.rows_pad;
+        const size_t want = (make_f32 ? elems * 4 : 0) + (make_bf16 ? elems * 2 : 0);
+        if (ctx->basis_bytes + want > kBasisBudgetBytes) {
+            FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // bases may be in use by enqueued kernels
+            free_bases(ctx);
+            b = Basis();
+            b.n_in = n_in; b.n_keep = n_keep; b.ld = (n_in + 63) / 64 * 64; b.rows_pad = (n_keep + 63) / 64 * 64;
+            it = ctx->bases.end();
+        }
+        float* pf = nullptr;
+        __nv_bfloat16* pb = nullptr;
+        if (need_f32 && !b.f32) FREQKV_CUDA(ctx, cudaMalloc(&pf, elems * 4));
+        if (need_bf16 && !b.bf16) {
+            const cudaError_t e = cudaMalloc(&pb, elems * 2);
+            if (e != cudaSuccess) {
+                if (pf) cudaFree(pf);
+                return cuda_fail(ctx, e, "cudaMalloc(basis)");
+            }
+        }
+        const cudaError_t e = launch_build_basis(pf, pb, n_in, n_keep, b.ld, b.rows_pad, stream);
+        if (e != cudaSuccess) {
+            if (pf) cudaFree(pf);
+            if (pb) cudaFree(pb);
+            return cuda_fail(ctx, e, "build_basis");
+        }
+        if (pf) { b.f32 = pf; ctx->basis_bytes += elems * 4; }
+        if (pb) { b.bf16 = pb; ctx->basis_bytes += elems * 2; }
+        ctx->bases[key] = b;
+    }
+    *out = b;
+    return FREQKV_OK;
+}
+
+freqkv_status get_scratch(freqkv_ctx* ctx, size_t bytes, void** out)
+{
+    if (bytes > ctx->scratch_bytes) {
+        if (ctx->scratch) {
+            FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // earlier launches may still read it
+            cudaFree(ctx->scratch);
+            ctx->scratch = nullptr;
+            ctx->scratch_bytes = 0;
+        }
+        FREQKV_CUDA(ctx, cudaMalloc(&ctx->scratch, bytes));
+        ctx->scratch_bytes = bytes;
+    }
+    *out = ctx->scratch;
+    return FREQKV_OK;
+}
+
+// Compress `count` sequences starting at batch0, all with the same (n_in, n_keep).
+freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, void* v, int32_t batch0,
+                             int32_t batch_count, int32_t n_in, int32_t n_keep, int32_t sink, int32_t variant,
+                             cudaStream_t stream)
+{
+    const CacheView view = make_view(l, k, v, batch0, batch_count);
+    const int32_t n_mat = 2 * view.mats_per_tensor;
+
+    if (variant == FREQKV_FDCT) {
+        FdctPlan plan;
+        const auto key = std::make_pair(n_in, n_keep);
+        auto it = ctx->fdct_plans.find(key);
+        if (it == ctx->fdct_plans.end()) {
+            const cudaError_t e = fdct_make_plan(n_in, n_keep, stream, &plan);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "fdct_make_plan");
+            ctx->fdct_plans[key] = plan;
+        } else {
+            plan = it->second;
+        }
+        const cudaError_t e = launch_fdct(view, l.dtype, n_mat, plan, sink, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "launch_fdct");
+        return FREQKV_OK;
+    }
+
+    Basis basis;
+    const bool gemm = variant == FREQKV_GEMM;
+    freqkv_status st = get_basis(ctx, n_in, n_keep, !gemm, gemm, stream, &basis);
+    if (st != FREQKV_OK) return st;
+
+    if (gemm) {
+        const cudaError_t e = launch_gemm(&ctx->gemm, view, l, k, v, batch0, batch_count, basis, sink, ctx->status_dev,
+                                          ctx->sm_count, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
+        return FREQKV_OK;
+    }
+
+    const size_t per_mat = (size_t)n_keep * l.head_dim * dtype_size(l.dtype);
+    int64_t chunk = (int64_t)std::max<size_t>(1, kScratchChunkBytes / per_mat);
+    chunk = std::min<int64_t>(chunk, n_mat);
+    chunk = std::min<int64_t>(chunk, 1 << 30);
+    void* scratch = nullptr;
+    st = get_scratch(ctx, (size_t)chunk * per_mat, &scratch);
+    if (st != FREQKV_OK) return st;
+    for (int32_t first = 0; first < n_mat; first += (int32_t)chunk) {
+        const int32_t count = (int32_t)std::min<int64_t>(chunk, n_mat - first);
+        cudaError_t e = launch_project_simt(view, l.dtype, first, count, basis, sink, scratch, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "project_simt");
+        e = launch_copy_back(view, l.dtype, first, count, n_keep, sink, scratch, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "copy_back");
+    }
+    return FREQKV_OK;
+}
+
+freqkv_status check_lengths(const freqkv_layout& l, int64_t cache_len, int64_t kept_len, int64_t sink)
+{
+    if (sink < 0 || cache_len < 0 || kept_len < 0) return FREQKV_ERR_INVALID_ARG;
+    if (sink > cache_len || cache_len > l.capacity) return FREQKV_ERR_INVALID_ARG;
+    if (kept_len > cache_len - sink) return FREQKV_ERR_INVALID_ARG;
+    return FREQKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+freqkv_status freqkv_layout_contiguous(freqkv_layout* out, freqkv_dtype dtype, int32_t batch, int32_t layers,
+                                       int32_t kv_heads, int32_t capacity, int32_t head_dim)
+{
+    if (!out) return FREQKV_ERR_INVALID_ARG;
+    out->dtype = dtype;
+    out->batch = batch;
+    out->layers = layers;
+    out->kv_heads = kv_heads;
+    out->capacity = capacity;
+    out->head_dim = head_dim;
+    out->stride_token = head_dim;
+    out->stride_head = (int64_t)capacity * head_dim;
+    out->stride_layer = out->stride_head * kv_heads;
+    out->stride_batch = out->stride_layer * layers;
+    return check_layout(out);
+}
+
+freqkv_status freqkv_create(freqkv_ctx** out, int device)
+{
+    if (!out) return FREQKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return FREQKV_ERR_CUDA;  // no CPU fallback
+    }
+    if (device < 0 || device >= n) return FREQKV_ERR_INVALID_ARG;
+    freqkv_ctx* ctx = new (std::nothrow) freqkv_ctx();
+    if (!ctx) return FREQKV_ERR_ALLOC;
+    ctx->device = device;
+    DeviceGuard g(device);
+    cudaDeviceProp prop;
+    if (!g.ok || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+        delete ctx;
+        return FREQKV_ERR_CUDA;
+    }
+    if (prop.major != 10) {  // kernels are built for sm_100a only
+        delete ctx;
+        return FREQKV_ERR_UNSUPPORTED;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&ctx->status_dev, sizeof(int32_t)) != cudaSuccess ||
+        cudaMemset(ctx->status_dev, 0, sizeof(int32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return FREQKV_ERR_ALLOC;
+    }
+    *out = ctx;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_destroy(freqkv_ctx* ctx)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    free_bases(ctx);
+    for (auto& kv : ctx->fdct_plans) fdct_free_plan(&kv.second);
+    gemm_release(&ctx->gemm);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->status_dev) cudaFree(ctx->status_dev);
+    cudaGetLastError();
+    delete ctx;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_set_variant(freqkv_ctx* ctx, freqkv_variant variant)
+{
+    if (!ctx || variant < FREQKV_AUTO || variant > FREQKV_SIMT) return FREQKV_ERR_INVALID_ARG;
+    ctx->forced = variant;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_resolve_variant(freqkv_ctx* ctx, const freqkv_layout* layout, int32_t n_in, int32_t n_keep,
+                                     int32_t* out_variant)
+{
+    if (!ctx || !out_variant) return FREQKV_ERR_INVALID_ARG;
+    const freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    if (n_in < 1 || n_keep < 1 || n_keep > n_in) return FREQKV_ERR_INVALID_ARG;
+    *out_variant = resolve(ctx, *layout, n_in, n_keep);
+    return *out_variant < 0 ? FREQKV_ERR_UNSUPPORTED : FREQKV_OK;
+}
+
+freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_dtype dtype, freqkv_variant variant,
+                          void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    if (n_in < 1 || n_keep < 1 || n_keep > n_in) return FREQKV_ERR_INVALID_ARG;
+    if (dtype != FREQKV_BF16 && dtype != FREQKV_F32) return FREQKV_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (variant == FREQKV_FDCT) {
+        if (!is_pow2(n_in) || !is_pow2(n_keep) || !fdct_supported(dtype, 128, n_in, n_keep)) return FREQKV_ERR_UNSUPPORTED;
+        const auto key = std::make_pair(n_in, n_keep);
+        if (ctx->fdct_plans.find(key) == ctx->fdct_plans.end()) {
+            FdctPlan plan;
+            const cudaError_t e = fdct_make_plan(n_in, n_keep, stream, &plan);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "fdct_make_plan");
+            ctx->fdct_plans[key] = plan;
+        }
+        return FREQKV_OK;
+    }
+    if (variant == FREQKV_GEMM && dtype != FREQKV_BF16) return FREQKV_ERR_UNSUPPORTED;
+    Basis b;
+    const bool gemm = variant == FREQKV_GEMM;
+    const bool both = variant == FREQKV_AUTO;
+    return get_basis(ctx, n_in, n_keep, !gemm || both, (gemm || both) && dtype == FREQKV_BF16, stream, &b);
+}
+
+freqkv_status freqkv_check_compress(const freqkv_layout* layout, const void* k, const void* v, int32_t cache_len,
+                                    int32_t kept_len, int32_t sink)
+{
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    st = check_tensors(*layout, k, v);
+    if (st != FREQKV_OK) return st;
+    return check_lengths(*layout, cache_len, kept_len, sink);
+}
+
+freqkv_status freqkv_check_append(const freqkv_layout* layout, const void* k, const void* v, const void* new_k,
+                                  const void* new_v, int32_t n_new, const int32_t* lens)
+{
+    if (!lens) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    st = check_tensors(*layout, k, v);
+    if (st != FREQKV_OK) return st;
+    if (n_new < 0) return FREQKV_ERR_INVALID_ARG;
+    if (n_new > 0 && (!new_k || !new_v)) return FREQKV_ERR_INVALID_ARG;
+    if (n_new > 0 && (((uintptr_t)new_k | (uintptr_t)new_v) & 15)) return FREQKV_ERR_UNSUPPORTED;
+    for (int32_t b = 0; b < layout->batch; ++b) {
+        if (lens[b] < 0 || lens[b] > layout->capacity) return FREQKV_ERR_INVALID_ARG;
+        if ((int64_t)lens[b] + n_new > layout->capacity) return FREQKV_ERR_CAPACITY;
+    }
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
+                              int32_t kept_len, int32_t sink, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = freqkv_check_compress(layout, k, v, cache_len, kept_len, sink);
+    if (st != FREQKV_OK) return st;
+    const int32_t n_in = cache_len - sink;
+    if (n_in == 0 || kept_len == 0 || kept_len == n_in) return FREQKV_OK;  // nothing to rewrite
+    const int32_t variant = resolve(ctx, *layout, n_in, kept_len);
+    if (variant < 0) return FREQKV_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
+                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t* lens,
+                                     const int32_t* kept_len, int32_t sink, void* cuda_stream)
+{
+    if (!ctx || !lens || !kept_len) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    st = check_tensors(*layout, k, v);
+    if (st != FREQKV_OK) return st;
+    std::vector<int32_t> variant(layout->batch, 0);
+    for (int32_t b = 0; b < layout->batch; ++b) {
+        st = check_lengths(*layout, lens[b], kept_len[b], sink);
+        if (st != FREQKV_OK) return st;
+        const int32_t n_in = lens[b] - sink;
+        if (n_in == 0 || kept_len[b] == 0 || kept_len[b] == n_in) continue;
+        variant[b] = resolve(ctx, *layout, n_in, kept_len[b]);
+        if (variant[b] < 0) return FREQKV_ERR_UNSUPPORTED;
+    }
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // Sequences are grouped by runs of equal (length, kept length); each run is one group.
+    for (int32_t b = 0; b < layout->batch;) {
+        int32_t e = b + 1;
+        while (e < layout->batch && lens[e] == lens[b] && kept_len[e] == kept_len[b]) ++e;
+        if (variant[b] > 0) {
+            st = compress_group(ctx, *layout, k, v, b, e - b, lens[b] - sink, kept_len[b], sink, variant[b], stream);
+            if (st != FREQKV_OK) return st;
+        }
+        b = e;
+    }
+    for (int32_t b = 0; b < layout->batch; ++b) lens[b] = sink + kept_len[b];
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
+                            const void* new_v, int32_t n_new, int32_t* lens, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    const freqkv_status st = freqkv_check_append(layout, k, v, new_k, new_v, n_new, lens);
+    if (st != FREQKV_OK) return st;
+    if (n_new == 0) return FREQKV_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    const CacheView view = make_view(*layout, k, v, 0, layout->batch);
+    const cudaError_t e =
+        launch_append(view, layout->dtype, layout->batch, lens, n_new, new_k, new_v, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "append");
+    for (int32_t b = 0; b < layout->batch; ++b) lens[b] += n_new;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int32_t word = 0;
+    FREQKV_CUDA(ctx, cudaMemcpyAsync(&word, ctx->status_dev, sizeof(word), cudaMemcpyDeviceToHost, stream));
+    FREQKV_CUDA(ctx, cudaMemsetAsync(ctx->status_dev, 0, sizeof(word), stream));
+    FREQKV_CUDA(ctx, cudaStreamSynchronize(stream));
+    if (word != 0) {
+        char buf[96];
+        snprintf(buf, sizeof(buf), "device status word 0x%08x (a bounded wait gave up)", (unsigned)word);
+        ctx->last_error = buf;
+        return FREQKV_ERR_TIMEOUT;
+    }
+    return FREQKV_OK;
+}
+
+const char* freqkv_last_error(freqkv_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+const char* freqkv_status_string(freqkv_status status)
+{
+    switch (status) {
+        case FREQKV_OK: return "FREQKV_OK";
+        case FREQKV_ERR_INVALID_ARG: return "FREQKV_ERR_INVALID_ARG";
+        case FREQKV_ERR_UNSUPPORTED: return "FREQKV_ERR_UNSUPPORTED";
+        case FREQKV_ERR_CAPACITY: return "FREQKV_ERR_CAPACITY";
+        case FREQKV_ERR_ALLOC: return "FREQKV_ERR_ALLOC";
+        case FREQKV_ERR_CUDA: return "FREQKV_ERR_CUDA";
+        case FREQKV_ERR_TIMEOUT: return "FREQKV_ERR_TIMEOUT";
+    }
+    return "FREQKV_ERR_UNKNOWN";
+}
+
+int32_t freqkv_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,60 @@
+// Projection basis of one compression (Section 3.3, Eq. 2-3 with the transforms of
+// Appendix A).  DCT-II of length N, truncation to L components, L-point inverse DCT and the
+// sqrt(L/N) rescale are one linear map Y = P X with
+//
+//   P[m][n] = (1/N) * [ 1 + 2 * sum_{t=1}^{L-1} cos(pi t (2m+1)/(2L)) * cos(pi t (2n+1)/(2N)) ].
+//
+// The product of cosines splits into cosines of the sum and difference angle, and each of the
+// two cosine series sums to a Dirichlet kernel:
+//
+//   P[m][n] = (1/(2N)) * [ D(a+) + D(a-) ],   a± = (2m+1) N ± (2n+1) L   (integers),
+//   D(a) = sin((2L-1) pi a / (4LN)) / sin(pi a / (4LN)),   D(0) = 2L-1.
+//
+// 0 < a+ < 4LN and |a-| < 2LN, so the denominator vanishes only at a- = 0.  The numerator's
+// phase is reduced exactly in 64-bit integers modulo 8LN before sinpi, so every entry is
+// accurate to a few fp64 ulps; it is rounded once to fp32 and once to bf16.
+#include "common.cuh"
+
+namespace freqkv {
+namespace {
+
+__device__ inline double dirichlet(int64_t a, int64_t L, int64_t LN4)
+{
+    if (a < 0) a = -a;  // D is even
+    if (a == 0) return (double)(2 * L - 1);
+    const int64_t r = ((2 * L - 1) * a) % (2 * LN4);
+    return sinpi((double)r / (double)LN4) / sinpi((double)a / (double)LN4);
+}
+
+__global__ void build_basis_kernel(float* __restrict__ p_f32, __nv_bfloat16* __restrict__ p_bf16, int32_t n_in,
+                                   int32_t n_keep, int32_t ld, int32_t rows_pad)
+{
+    const int64_t total = (int64_t)rows_pad * ld;
+    const int64_t N = n_in, L = n_keep, LN4 = 4 * L * N;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = i / ld, n = i % ld;
+        double p = 0.0;
+        if (m < L && n < N) {
+            const int64_t u = (2 * m + 1) * N, w = (2 * n + 1) * L;
+            p = (dirichlet(u + w, L, LN4) + dirichlet(u - w, L, LN4)) / (double)(2 * N);
+        }
+        if (p_f32) p_f32[i] = (float)p;
+        if (p_bf16) p_bf16[i] = __double2bfloat16(p);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
+                               int32_t rows_pad, cudaStream_t stream)
+{
+    const int64_t total = (int64_t)rows_pad * ld;
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks < 1) blocks = 1;
+    build_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(p_f32, p_bf16, n_in, n_keep, ld, rows_pad);
+    return cudaGetLastError();
+}
+
+}  // namespace freqkv

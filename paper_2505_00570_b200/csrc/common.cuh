@@ -1,0 +1,64 @@
+// Shared declarations of the FreqKV CUDA library (internal; the public surface is
+// include/freqkv.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "freqkv.h"
+
+namespace freqkv {
+
+// Device-side view of the K and V caches: matrix i of a call is tensor i / mats_per_tensor
+// (0 = K, 1 = V), and inside the tensor (batch, layer, kv_head) in row-major order.
+struct CacheView {
+    void* base[2];
+    int64_t stride_batch, stride_layer, stride_head, stride_token;  // elements
+    int32_t layers, kv_heads, head_dim;
+    int32_t mats_per_tensor;  // batch * layers * kv_heads
+    int32_t batch0;           // first batch index covered (ragged calls address one sequence)
+};
+
+__host__ __device__ inline int64_t matrix_offset(const CacheView& v, int32_t idx_in_tensor)
+{
+    const int32_t h = idx_in_tensor % v.kv_heads;
+    const int32_t l = (idx_in_tensor / v.kv_heads) % v.layers;
+    const int32_t b = idx_in_tensor / (v.kv_heads * v.layers) + v.batch0;
+    return (int64_t)b * v.stride_batch + (int64_t)l * v.stride_layer + (int64_t)h * v.stride_head;
+}
+
+__host__ __device__ inline void* tensor_base(const CacheView& v, int32_t tensor)
+{
+    return tensor ? v.base[1] : v.base[0];  // a select, not an indexed load of the parameter struct
+}
+
+// Projection basis of one (n_in, n_keep) pair: P[m][n], row-major with leading dimension ld,
+// rows padded to rows_pad and columns to ld with zeros.
+struct Basis {
+    float* f32 = nullptr;          // SIMT path
+    __nv_bfloat16* bf16 = nullptr; // tensor-core path
+    int32_t n_in = 0, n_keep = 0, ld = 0, rows_pad = 0;
+};
+
+// ---- kernel launchers (each returns the cudaError_t of its launch) ----
+
+// P[m][n] for m < n_keep, n < n_in from the closed form; zero padding elsewhere.
+cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
+                               int32_t rows_pad, cudaStream_t stream);
+
+// scratch[i - first][m][c] = sum_n P[m][n] * X_i[sink + n][c] for matrices first .. first+count-1.
+cudaError_t launch_project_simt(const CacheView& view, int32_t dtype, int32_t first, int32_t count, const Basis& basis,
+                                int32_t sink, void* scratch, cudaStream_t stream);
+
+// cache rows [sink, sink + n_keep) of matrices first .. first+count-1 <- scratch.
+cudaError_t launch_copy_back(const CacheView& view, int32_t dtype, int32_t first, int32_t count, int32_t n_keep,
+                             int32_t sink, const void* scratch, cudaStream_t stream);
+
+// rows [lens[b], lens[b] + n_new) of every matrix <- new rows.
+cudaError_t launch_append(const CacheView& view, int32_t dtype, int32_t batch, const int32_t* lens_host,
+                          int32_t n_new, const void* new_k, const void* new_v, cudaStream_t stream);
+
+inline size_t dtype_size(int32_t dtype) { return dtype == FREQKV_F32 ? 4 : 2; }
+
+}  // namespace freqkv

@@ -1,0 +1,84 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI on a seeded
+cache surrounded by canaries and compare it with the CPU oracle on the same bits."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2505_00570_b200 import binding as fk
+from paper_2505_00570_b200 import synth
+
+TOL = {torch.float32: 1e-5, torch.bfloat16: 1e-2}  # max per-matrix relative L2 (spec bars)
+GUARD = 4096  # canary elements before and after each tensor
+
+
+def guarded_cache(w: synth.Workload, device, fill_len=None, row_pad: int = 0, batch=None):
+    """K and V as views into larger buffers: canaries before and after, and (row_pad > 0)
+    padding elements after every row, all of which must survive a call bit for bit."""
+    k0, v0 = synth.make_cache(w, device, fill_len=fill_len, batch=batch)
+    out = []
+    for t in (k0, v0):
+        B, Ly, H, cap, hd = t.shape
+        st = hd + row_pad
+        n = B * Ly * H * cap * st
+        buf = torch.empty(n + 2 * GUARD, dtype=t.dtype, device=device)
+        buf.fill_(-7.0)  # canary value
+        view = buf[GUARD:GUARD + n].view(B, Ly, H, cap, st)[..., :hd]
+        view.copy_(t)
+        out.append((buf, view))
+    return out[0], out[1]
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def rel_l2(got: np.ndarray, want: np.ndarray) -> float:
+    return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def check_compress(ctx: fk.Context, w: synth.Workload, cache_len: int, kept_len: int, sink: int, variant: int,
+                   row_pad: int = 0, sample: int | None = None, batch=None):
+    """Compress on the GPU, then check (1) every byte outside rows [sink, sink+kept_len) is
+    unchanged, canaries and padding included, (2) the rewritten rows match the oracle matrix by
+    matrix within the tolerance of the dtype.  Returns the worst relative L2."""
+    dev = torch.device("cuda", ctx.device)
+    (kbuf, k), (vbuf, v) = guarded_cache(w, dev, fill_len=cache_len, row_pad=row_pad, batch=batch)
+    kbuf0, vbuf0 = kbuf.clone(), vbuf.clone()
+    k_in, v_in = k.clone(), v.clone()
+    ctx.set_variant(variant)
+    new_len = ctx.compress(k, v, cache_len, kept_len, sink)
+    assert ctx.last_device_status() == fk.OK
+    assert new_len == sink + kept_len
+
+    # (1) bit-exact outside the rewritten rows
+    for buf, buf0, t in ((kbuf, kbuf0, k), (vbuf, vbuf0, v)):
+        mask_src = torch.zeros_like(t, dtype=torch.bool)
+        mask_src[..., sink:sink + kept_len, :] = True
+        B, Ly, H, cap, hd = t.shape
+        st = hd + row_pad
+        full = torch.zeros(buf.numel(), dtype=torch.bool, device=dev)
+        full[GUARD:GUARD + B * Ly * H * cap * st].view(B, Ly, H, cap, st)[..., :hd].copy_(mask_src)
+        raw, raw0 = buf.view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32), \
+            buf0.view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32)
+        assert torch.equal(raw[~full], raw0[~full]), "bytes outside rows [sink, sink+kept_len) changed"
+
+    # (2) oracle parity on all (or a seeded sample of) matrices
+    n_mat = 2 * k.shape[0] * k.shape[1] * k.shape[2]
+    ids = range(n_mat) if sample is None else synth.sample_matrix_ids(n_mat, sample, w.seed + 5)
+    worst = 0.0
+    n_in = cache_len - sink
+    per = n_mat // 2
+    for i in ids:
+        t_in, t_out = (k_in, k) if i < per else (v_in, v)
+        j = i % per
+        b, l, h = j // (k.shape[1] * k.shape[2]), (j // k.shape[2]) % k.shape[1], j % k.shape[2]
+        x = to_f64(t_in[b, l, h, sink:sink + n_in])
+        want = oracle.compress_matrix(x, kept_len)
+        got = to_f64(t_out[b, l, h, sink:sink + kept_len])
+        if kept_len == n_in:
+            assert np.array_equal(got, x)  # identity must be bit-exact
+        worst = max(worst, rel_l2(got, want))
+    assert worst <= TOL[w.dtype], f"relative L2 {worst:.3e} exceeds {TOL[w.dtype]:.0e}"
+    return worst

@@ -1,0 +1,161 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the
+same seeded inputs.  Tolerances: relative L2 <= 1e-5 (fp32 caches), <= 1e-2 (bf16 caches),
+worst matrix; every byte outside the rewritten rows bit-exact."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_00570_b200 import binding as fk
+from paper_2505_00570_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = fk.Context(0)
+    yield c
+    c.close()
+
+
+def small(name="t", B=1, Ly=2, H=2, hd=128, cap=512, dtype=torch.float32, sink=0, rho=0.9, outliers=0, seed=7):
+    return synth.Workload(name, B, Ly, H, hd, cap, dtype, sink, rho, outliers, synth.BASE_SEED + seed)
+
+
+# ---- config 1: tiny single-head fp32, 512 -> 256, no sinks
+def test_config1_tiny_fp32(ctx):
+    w = synth.WORKLOADS["tiny"]
+    worst = parity.check_compress(ctx, w, 512, 256, 0, fk.AUTO)
+    assert worst < 1e-5
+
+
+@pytest.mark.parametrize("variant", [fk.SIMT])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n_in,kept", [(1, 1), (2, 1), (3, 2), (5, 2), (8, 4), (31, 15), (62, 31), (127, 63),
+                                        (128, 64), (129, 64), (300, 150), (500, 125), (508, 381)])
+def test_small_lengths(ctx, variant, dtype, n_in, kept):
+    sink = 4
+    w = small(cap=n_in + sink + 3, dtype=dtype, sink=sink, outliers=2 if dtype == torch.bfloat16 else 0)
+    parity.check_compress(ctx, w, n_in + sink, kept, sink, variant)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_row_padding_and_canaries(ctx, dtype):
+    w = small(cap=200, dtype=dtype, sink=4, B=2)
+    parity.check_compress(ctx, w, 197, 96, 4, fk.SIMT, row_pad=8)
+
+
+@pytest.mark.parametrize("hd", [64, 96, 256])
+def test_other_head_dims(ctx, hd):
+    w = small(cap=160, hd=hd, dtype=torch.bfloat16, sink=2)
+    parity.check_compress(ctx, w, 150, 74, 2, fk.SIMT)
+
+
+def test_degenerate_cases_write_nothing(ctx):
+    w = small(cap=64, dtype=torch.bfloat16, sink=4)
+    parity.check_compress(ctx, w, 64, 60, 4, fk.AUTO)   # identity
+    parity.check_compress(ctx, w, 64, 0, 4, fk.AUTO)    # keep nothing
+    parity.check_compress(ctx, w, 4, 0, 4, fk.AUTO)     # only sinks in the cache
+
+
+def test_invalid_arguments_raise(ctx):
+    k = torch.zeros(1, 1, 1, 64, 128, device="cuda", dtype=torch.bfloat16)
+    v = torch.zeros_like(k)
+    with pytest.raises(fk.FreqKVError) as e:
+        ctx.compress(k, v, 64, 61, 4)
+    assert e.value.status == fk.ERR_INVALID_ARG
+    with pytest.raises(fk.FreqKVError):
+        ctx.compress(k, k, 64, 30, 4)
+    with pytest.raises(fk.FreqKVError):
+        ctx.compress(k, v.float(), 64, 30, 4)
+
+
+# ---- config 2 shapes (LLaMA-2-7B: 4092 -> 2046, 4 sinks), a few heads, sampled matrices
+def test_config2_shape_simt(ctx):
+    w = dataclasses.replace(synth.WORKLOADS["llama2_7b"], layers=1, kv_heads=4)
+    parity.check_compress(ctx, w, 4096, 2046, 4, fk.SIMT, sample=4)
+
+
+# ---- append, the lazy trigger and a short iterative stream against the oracle
+def test_append_rows_and_capacity(ctx):
+    w = small(cap=40, dtype=torch.bfloat16, B=3, sink=4)
+    k, v = synth.make_cache(w, "cuda", fill_len=0)
+    k.fill_(1.5), v.fill_(-2.5)
+    k0, v0 = k.clone(), v.clone()
+    nk = torch.randn(3, 2, 2, 5, 128, device="cuda").to(torch.bfloat16)
+    nv = torch.randn(3, 2, 2, 5, 128, device="cuda").to(torch.bfloat16)
+    lens = ctx.append(k, v, nk, nv, [0, 7, 35])
+    assert lens == [5, 12, 40]
+    for b, start in enumerate([0, 7, 35]):
+        assert torch.equal(k[b, :, :, start:start + 5], nk[b]) and torch.equal(v[b, :, :, start:start + 5], nv[b])
+        keep = torch.ones(40, dtype=torch.bool)
+        keep[start:start + 5] = False
+        assert torch.equal(k[b][:, :, keep], k0[b][:, :, keep]) and torch.equal(v[b][:, :, keep], v0[b][:, :, keep])
+    with pytest.raises(fk.FreqKVError) as e:
+        ctx.append(k, v, nk, nv, [5, 12, 36])
+    assert e.value.status == fk.ERR_CAPACITY
+    assert torch.equal(k[2, :, :, 35:40], nk[2])  # a refused append wrote nothing
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_iterative_stream_matches_oracle(ctx, dtype):
+    """Tokens enter one at a time; a full cache is compressed to half its non-sink length
+    before the next token goes in (Section 3.4).  The GPU cache is compared with the oracle's
+    replay of the same stream after every compression."""
+    cap, S, T, hd = 48, 4, 200, 64
+    w = small(cap=cap, hd=hd, dtype=dtype, sink=S, Ly=1, H=2, B=2)
+    ctx.set_variant(fk.AUTO)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    scales = synth.channel_scales(w, gen, "cuda")
+    k, v = synth.make_cache(w, "cuda", fill_len=0)
+    toks_k, state_k = synth.ar1_rows(w, T, gen, "cuda", scales)
+    toks_v, state_v = synth.ar1_rows(w, T, gen, "cuda", scales)
+    lens = [0, 0]
+    L = (cap - S) // 2
+    count = 0
+    for t in range(T):
+        try:
+            lens = ctx.append(k, v, toks_k[:, :, :, t:t + 1].contiguous(), toks_v[:, :, :, t:t + 1].contiguous(), lens)
+        except fk.FreqKVError as e:
+            assert e.status == fk.ERR_CAPACITY
+            new_len = ctx.compress(k, v, cap, L, S)
+            lens = [new_len, new_len]
+            count += 1
+            lens = ctx.append(k, v, toks_k[:, :, :, t:t + 1].contiguous(), toks_v[:, :, :, t:t + 1].contiguous(), lens)
+    assert count == oracle.compression_count(T, cap, S, L)
+    # oracle replay: it compresses its own fp64 state, so the gap grows with the number of
+    # compressions by at most one rounding of the cache dtype each time
+    tol = {torch.float32: 1e-5, torch.bfloat16: 1e-2}[dtype] * max(1, count) ** 0.5
+    for b in range(2):
+        for h in range(2):
+            for cache_t, toks in ((k, toks_k), (v, toks_v)):
+                want, n, c = oracle.stream(parity.to_f64(toks[b, 0, h]), cap, S, 0.5)
+                assert n == lens[b] and c == count
+                got = parity.to_f64(cache_t[b, 0, h, :n])
+                assert np.array_equal(got[:S], want[:S])
+                assert parity.rel_l2(got, want[:n]) < tol
+
+
+def test_ragged_batch_small(ctx):
+    """Sequences of different lengths, each compressed to half its own non-sink length."""
+    w = small(cap=300, dtype=torch.bfloat16, sink=4, B=4, Ly=1, H=2, outliers=2)
+    k, v = synth.make_cache(w, "cuda")
+    k_in, v_in = k.clone(), v.clone()
+    lens = [300, 41, 177, 177]
+    kept = [(n - 4) // 2 for n in lens]
+    ctx.set_variant(fk.AUTO)
+    new_lens = ctx.compress_ragged(k, v, lens, kept, 4)
+    assert new_lens == [4 + x for x in kept]
+    for b in range(4):
+        for h in range(2):
+            for t_in, t_out in ((k_in, k), (v_in, v)):
+                want = oracle.compress_matrix(parity.to_f64(t_in[b, 0, h, 4:lens[b]]), kept[b])
+                got = parity.to_f64(t_out[b, 0, h, 4:4 + kept[b]])
+                assert parity.rel_l2(got, want) < 1e-2
+                assert torch.equal(t_out[b, 0, h, :4], t_in[b, 0, h, :4])
+                assert torch.equal(t_out[b, 0, h, 4 + kept[b]:], t_in[b, 0, h, 4 + kept[b]:])

@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the FreqKV hot path on B200: KV-compress GB/s of cache in.
+
+One *step* is one pass of the whole hot path over one batch of synthetic input, as in the
+chunk-wise loop of Section 3.4: the cache is full, so the incoming chunk is refused
+(``FREQKV_ERR_CAPACITY``, the lazy trigger), every K and V matrix is compressed in place
+(DCT-II -> keep L -> L-point IDCT -> rescale, sinks untouched), and the chunk of
+``capacity - sink - L`` new rows is appended, which fills the cache again for the next step.
+
+``value`` = (bytes of cache in per step) / (device time per step), inputs resident in HBM.
+``e2e``   = the same metric through ``freqkv_compress_host`` with the cache in pinned host
+            memory (host->device and device->host copies inside the timed region).
+``roofline`` describes the dominant kernel (the transform), timed with CUDA events recorded by
+the library around that launch on the launching stream.
+
+Launch: ``python bench.py --gpus N --steps K --warmup W``; for N > 1 under
+``python -m torch.distributed.run --nproc-per-node N``: the path has no exchange step, so N
+ranks are N independent replicas (weak scaling, no collective on the data path).
+``--impl reference`` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "KV-compress GB/s of cache in (7B shape, 4096->2048) and % of roofline"
+UNIT = "GB/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def load_traffic(workload: str, variant: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        table = json.load(f)
+    return table.get(f"{workload}:{variant}")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._period = period_s
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self._nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report that, do not fail the bench
+            self._nv = None
+            self.error = repr(e)
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or getattr(
+            nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = get_reasons(self._h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+               "samples": len(self.samples)}
+        if self.samples:
+            s = sorted(self.samples)
+            out["sm_mhz"] = s[len(s) // 2]
+        if self._nv is None:
+            out["error"] = getattr(self, "error", "nvml unavailable")
+        return out
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(ms: float, device) -> float:
+    """Slowest rank's time (replicas run side by side; the job is as slow as its slowest)."""
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+def workload_numbers(w, cache_len, kept, sink):
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    m = w.n_matrices
+    n_in = cache_len - sink
+    return {
+        "matrices": m,
+        "cache_in_bytes": m * cache_len * w.head_dim * e,
+        "algorithmic_bytes": m * (n_in + kept) * w.head_dim * e,   # read N' rows, write L rows
+        "projection_flops": 2.0 * kept * n_in * w.head_dim * m,    # what the basis GEMM executes
+        "append_bytes": 2 * m * (cache_len - sink - kept) * w.head_dim * e,
+    }
+
+
+def run_reference(args, rank):
+    """CPU oracle arm: each step compresses a bounded sample (one matrix) of the workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2505_00570_b200 import synth
+    import dataclasses
+
+    w = synth.WORKLOADS[args.workload]
+    cache_len, sink = w.capacity, w.sink
+    kept = w.kept_len(cache_len)
+    one = dataclasses.replace(w, batch=1, layers=1, kv_heads=1)
+    k, _ = synth.make_cache(one, "cpu")
+    x = k[0, 0, 0, sink:cache_len].to(torch.float64).numpy()
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    bytes_in = cache_len * w.head_dim * e
+    for _ in range(args.warmup):
+        oracle.compress_matrix(x, kept)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.compress_matrix(x, kept)
+    dt = time.perf_counter() - t0
+    val = bytes_in * args.steps / dt / 1e9
+    cores = oracle.threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "cache_len": cache_len, "kept_len": kept, "sink": sink,
+                   "sample": "1 of %d matrices per step" % w.n_matrices},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "one %dx%d matrix per step, %d steps" % (cache_len - sink, w.head_dim, args.steps)},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(w, k, v, cache_len, kept, sink, budget_s=12.0):
+    """The oracle, as it stands, on a bounded sample of this workload's matrices."""
+    import oracle
+
+    e = 2 if w.dtype == torch.bfloat16 else 4
+    flat = k.view(-1, k.shape[-2], k.shape[-1])
+    x0 = flat[0, sink:cache_len].to("cpu").to(torch.float64).numpy()
+    t0 = time.perf_counter()
+    oracle.compress_matrix(x0, kept)
+    one = time.perf_counter() - t0
+    count = int(max(2, min(64, budget_s / max(one, 1e-3))))
+    ids = torch.linspace(0, flat.shape[0] - 1, count).long().tolist()
+    xs = [flat[i, sink:cache_len].to("cpu").to(torch.float64).numpy() for i in ids]
+    t0 = time.perf_counter()
+    for x in xs:
+        oracle.compress_matrix(x, kept)
+    dt = time.perf_counter() - t0
+    return {"value": count * cache_len * w.head_dim * e / dt / 1e9, "unit": UNIT, "cores": oracle.threads(),
+            "kind": "oracle", "sample": "%d of %d matrices (%dx%d -> %d rows), %.1f s" %
+            (count, w.n_matrices, cache_len - sink, w.head_dim, kept, dt)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b")
+    ap.add_argument("--variant", default="auto", choices=["auto", "gemm", "fdct", "simt"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank, local_rank, world = dist_env()
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    from paper_2505_00570_b200 import binding as fk
+    from paper_2505_00570_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    n_gpus = world
+
+    w = synth.WORKLOADS[args.workload]
+    cache_len, sink = w.capacity, w.sink
+    kept = w.kept_len(cache_len)
+    n_new = cache_len - sink - kept
+    nums = workload_numbers(w, cache_len, kept, sink)
+
+    ctx = fk.Context(local_rank)
+    variant = {"auto": fk.AUTO, "gemm": fk.GEMM, "fdct": fk.FDCT, "simt": fk.SIMT}[args.variant]
+    ctx.set_variant(variant)
+    k, v = synth.make_cache(w, dev, seed_offset=rank)
+    lay = fk.layout_of(k)
+    chosen = ctx.resolve_variant(lay, cache_len - sink, kept)
+    if chosen < 0:
+        raise SystemExit(f"variant {args.variant} cannot run {args.workload}")
+    chosen_name = fk.VARIANT_NAMES[chosen]
+    base = cpu_baseline(w, k, v, cache_len, kept, sink) if (rank == 0 and n_gpus == 1 and not args.no_cpu_baseline) else None
+
+    # the incoming chunk: the first n_new rows of a second seeded draw, resident in HBM
+    nk = k[:, :, :, :n_new].flip(3).contiguous()
+    nv = v[:, :, :, :n_new].flip(3).contiguous()
+    lens = [cache_len] * w.batch
+
+    def step(lens):
+        try:
+            return ctx.append(k, v, nk, nv, lens)        # refused while the cache is full
+        except fk.FreqKVError as err:
+            if err.status != fk.ERR_CAPACITY:
+                raise
+        new_len = ctx.compress(k, v, cache_len, kept, sink)
+        return ctx.append(k, v, nk, nv, [new_len] * w.batch)
+
+    for _ in range(args.warmup):
+        lens = step(lens)
+    torch.cuda.synchronize()
+    if ctx.last_device_status() != fk.OK:
+        raise SystemExit("device status reported an error during warm-up")
+    ctx.get_timing()
+    _, _, launches0 = ctx.get_timing()
+    ctx.set_timing(True)
+
+    sampler = ClockSampler(local_rank)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for _ in range(args.steps):
+        lens = step(lens)
+    stop.record()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(start.elapsed_time(stop), dev)
+    t_launches, t_ms, launches1 = ctx.get_timing()
+    ctx.set_timing(False)
+    status = ctx.last_device_status()
+    if status != fk.OK:
+        raise SystemExit("device status reported an error in the timed region")
+    ms_step = ms_total / args.steps
+    value = n_gpus * nums["cache_in_bytes"] / (ms_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the transform launch)
+    peaks = load_peaks()
+    kernel_ms = t_ms / max(t_launches, 1)
+    if chosen == fk.GEMM:
+        achieved = nums["projection_flops"] / (kernel_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": "sustained, of " + peaks["source"],
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"]}
+    elif chosen == fk.FDCT:
+        achieved = nums["algorithmic_bytes"] / (kernel_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_kind": "copy, of " + peaks["source"]}
+    else:
+        # fp32 FFMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        achieved = nums["projection_flops"] / (kernel_ms * 1e-3) / 1e12
+        roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_kind": "fp32 FFMA, derived from unit counts and max clock"}
+    roof["kernel"] = chosen_name
+    roof["kernel_ms"] = kernel_ms
+    roof["traffic"] = load_traffic(args.workload, chosen_name)
+
+    # ---- end to end through the host-buffer entry point (rank-local pinned host cache)
+    e2e = None
+    if args.e2e_steps > 0:
+        kh = torch.empty(k.shape, dtype=k.dtype, pin_memory=True)
+        vh = torch.empty(v.shape, dtype=v.dtype, pin_memory=True)
+        kh.copy_(k), vh.copy_(v)
+        torch.cuda.synchronize()
+        h2d = d2h = 0
+        for i in range(1 + args.e2e_steps):
+            if i == 1:
+                barrier()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+            _, h2d, d2h = ctx.compress_host(kh, vh, cache_len, kept, sink)
+            torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        dt_ms = max_over_ranks(dt * 1e3 / args.e2e_steps, dev)
+        e2e = {"value": n_gpus * nums["cache_in_bytes"] / (dt_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": dt_ms, "steps": args.e2e_steps,
+               "call": "freqkv_compress_host, cache in pinned host memory"}
+        del kh, vh
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": n_gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": w.batch, "layers": w.layers, "kv_heads": w.kv_heads,
+                       "head_dim": w.head_dim, "capacity": w.capacity, "cache_len": cache_len, "sink": sink,
+                       "kept_len": kept, "appended_rows_per_step": n_new, "variant": chosen_name,
+                       "l2": "inputs larger than L2 (%.2f GB of cache per step)" % (nums["cache_in_bytes"] / 1e9),
+                       "parallelism": "replicas only" if n_gpus > 1 else "single GPU",
+                       "step": "refused append (lazy trigger) + compress K,V in place + append chunk"},
+            "compress_only": {"ms": kernel_ms, "cache_in_GBps": nums["cache_in_bytes"] / (kernel_ms * 1e-3) / 1e9},
+            "roofline": roof, "cpu_baseline": base, "e2e": e2e, "clocks": clocks,
+            "gpu_launches": launches1 - launches0,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -123,6 +123,28 @@ freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layou
 freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
                             const void* new_v, int32_t n_new, int32_t* lens, void* cuda_stream);
 
+/* Host-buffer form of freqkv_compress for callers whose cache lives in host memory (pinned
+ * memory gives full copy bandwidth; pageable memory works).  k_host / v_host use `layout` in
+ * host memory.  Rows [sink, cache_len) of every matrix are copied to a device staging cache the
+ * context owns (allocated on first use, same layout), compressed there exactly as
+ * freqkv_compress does, and rows [sink, sink+kept_len) are copied back over the host rows.
+ * All copies and kernels are enqueued on `cuda_stream`; the host buffers must stay valid and
+ * untouched until that stream has been synchronised.  h2d_bytes / d2h_bytes (optional, may be
+ * NULL) receive the bytes moved each way. */
+freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout, void* k_host, void* v_host,
+                                   int32_t cache_len, int32_t kept_len, int32_t sink, void* cuda_stream,
+                                   int64_t* h2d_bytes, int64_t* d2h_bytes);
+
+/* Instrumentation for benchmarks.  With timing enabled every compression records a CUDA event
+ * pair on the caller's stream around its transform kernel (the projection / fast-transform
+ * launch, not the copy-back or table builders).  freqkv_get_timing waits for the recorded
+ * events, returns the number of timed transform launches and their summed device time in
+ * milliseconds since the last call, plus the number of kernels of any kind this context has
+ * launched since creation, and resets the timing sums.  Any output pointer may be NULL. */
+freqkv_status freqkv_set_timing(freqkv_ctx* ctx, int32_t enabled);
+freqkv_status freqkv_get_timing(freqkv_ctx* ctx, int64_t* transform_launches, double* transform_ms,
+                                int64_t* kernels_launched);
+
 /* Synchronise `cuda_stream`, then read and clear the device status word.  FREQKV_OK unless a
  * kernel's bounded wait (mbarrier / flag) ran out, in which case the affected output rows are
  * undefined and FREQKV_ERR_TIMEOUT is returned; the context stays usable. */

@@ -25,7 +25,8 @@ EXPORTS = [
     "freqkv_layout_contiguous", "freqkv_create", "freqkv_destroy", "freqkv_set_variant",
     "freqkv_resolve_variant", "freqkv_plan", "freqkv_compress", "freqkv_compress_ragged",
     "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
-    "freqkv_last_error", "freqkv_status_string", "freqkv_version",
+    "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
+    "freqkv_set_timing", "freqkv_get_timing",
 ]
 
 
@@ -70,6 +71,10 @@ def lib() -> ctypes.CDLL:
         L.freqkv_last_device_status.argtypes = [c_void_p, c_void_p]
         L.freqkv_check_compress.argtypes = [LP, c_void_p, c_void_p, c_int32, c_int32, c_int32]
         L.freqkv_check_append.argtypes = [LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P]
+        L.freqkv_compress_host.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
+                                           POINTER(c_int64), POINTER(c_int64)]
+        L.freqkv_set_timing.argtypes = [c_void_p, c_int32]
+        L.freqkv_get_timing.argtypes = [c_void_p, POINTER(c_int64), POINTER(ctypes.c_double), POINTER(c_int64)]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -206,6 +211,31 @@ class Context:
                                  new_v.data_ptr(), n_new, c_lens, _stream_ptr(stream))
         self._check(st, "freqkv_append")
         return list(c_lens)
+
+    def compress_host(self, k_host: torch.Tensor, v_host: torch.Tensor, cache_len: int, kept_len: int, sink: int,
+                      stream=None) -> tuple[int, int, int]:
+        """Host-buffer form: K and V live in (pinned) host memory; the library copies the
+        non-sink rows in, compresses on the device and copies the kept rows back, all enqueued
+        on the stream.  Returns (new length, bytes host->device, bytes device->host)."""
+        if k_host.is_cuda or v_host.is_cuda:
+            raise FreqKVError(ERR_INVALID_ARG, "compress_host takes host tensors")
+        lay = layout_of(k_host)
+        if tuple(v_host.shape) != tuple(k_host.shape) or v_host.stride() != k_host.stride() or v_host.dtype != k_host.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        h2d, d2h = c_int64(0), c_int64(0)
+        st = lib().freqkv_compress_host(self._h, ctypes.byref(lay), k_host.data_ptr(), v_host.data_ptr(), cache_len,
+                                        kept_len, sink, _stream_ptr(stream), ctypes.byref(h2d), ctypes.byref(d2h))
+        self._check(st, "freqkv_compress_host")
+        return sink + kept_len, h2d.value, d2h.value
+
+    def set_timing(self, enabled: bool):
+        self._check(lib().freqkv_set_timing(self._h, 1 if enabled else 0), "freqkv_set_timing")
+
+    def get_timing(self) -> tuple[int, float, int]:
+        """(timed transform launches, their summed device ms, kernels launched since creation)."""
+        n, ms, k = c_int64(0), ctypes.c_double(0.0), c_int64(0)
+        self._check(lib().freqkv_get_timing(self._h, ctypes.byref(n), ctypes.byref(ms), ctypes.byref(k)), "freqkv_get_timing")
+        return n.value, ms.value, k.value
 
     def last_device_status(self, stream=None) -> int:
         return lib().freqkv_last_device_status(self._h, _stream_ptr(stream))

@@ -29,6 +29,13 @@ struct freqkv_ctx {
     int32_t* status_dev = nullptr;
     GemmState gemm;
     std::string last_error;
+    // instrumentation
+    bool timing = false;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> pending, spare;
+    int64_t kernels_launched = 0;
+    // host-buffer entry point: device staging caches
+    void* stage[2] = {nullptr, nullptr};
+    size_t stage_bytes = 0;
 };
 
 namespace {
@@ -205,6 +212,7 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need
             if (pb) cudaFree(pb);
             return cuda_fail(ctx, e, "build_basis");
         }
+        ctx->kernels_launched += 1;
         if (pf) { b.f32 = pf; ctx->basis_bytes += elems * 4; }
         if (pb) { b.bf16 = pb; ctx->basis_bytes += elems * 2; }
         ctx->bases[key] = b;
@@ -229,6 +237,38 @@ freqkv_status get_scratch(freqkv_ctx* ctx, size_t bytes, void** out)
     return FREQKV_OK;
 }
 
+struct TransformTimer {
+    freqkv_ctx* ctx;
+    cudaStream_t stream;
+    std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
+    TransformTimer(freqkv_ctx* c, cudaStream_t s) : ctx(c), stream(s) { begin(); }
+    TransformTimer(freqkv_ctx* c, cudaStream_t s, bool start_now) : ctx(c), stream(s)
+    {
+        if (start_now) begin();
+    }
+    void begin()
+    {
+        if (!ctx->timing) return;
+        if (!ctx->spare.empty()) {
+            ev = ctx->spare.back();
+            ctx->spare.pop_back();
+        } else if (cudaEventCreate(&ev.first) != cudaSuccess || cudaEventCreate(&ev.second) != cudaSuccess) {
+            ev = {nullptr, nullptr};
+            cudaGetLastError();
+            return;
+        }
+        cudaEventRecord(ev.first, stream);
+    }
+    void end()
+    {
+        if (!ev.first) return;
+        cudaEventRecord(ev.second, stream);
+        ctx->pending.push_back(ev);
+        ev = {nullptr, nullptr};
+    }
+    ~TransformTimer() { end(); }
+};
+
 // Compress `count` sequences starting at batch0, all with the same (n_in, n_keep).
 freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, void* v, int32_t batch0,
                              int32_t batch_count, int32_t n_in, int32_t n_keep, int32_t sink, int32_t variant,
@@ -248,8 +288,13 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
         } else {
             plan = it->second;
         }
-        const cudaError_t e = launch_fdct(view, l.dtype, n_mat, plan, sink, stream);
+        cudaError_t e;
+        {
+            TransformTimer timer(ctx, stream);
+            e = launch_fdct(view, l.dtype, n_mat, plan, sink, stream);
+        }
         if (e != cudaSuccess) return cuda_fail(ctx, e, "launch_fdct");
+        ctx->kernels_launched += 1;
         return FREQKV_OK;
     }
 
@@ -259,9 +304,15 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
     if (st != FREQKV_OK) return st;
 
     if (gemm) {
+        TransformTimer timer(ctx, stream, false);
+        LaunchHooks hooks;
+        hooks.user = &timer;
+        hooks.before = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->begin(); };
+        hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
         const cudaError_t e = launch_gemm(&ctx->gemm, view, l, k, v, batch0, batch_count, basis, sink, ctx->status_dev,
-                                          ctx->sm_count, stream);
+                                          ctx->sm_count, hooks, stream);
         if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
+        ctx->kernels_launched += ctx->gemm.kernels_last_call;
         return FREQKV_OK;
     }
 
@@ -274,10 +325,15 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
     if (st != FREQKV_OK) return st;
     for (int32_t first = 0; first < n_mat; first += (int32_t)chunk) {
         const int32_t count = (int32_t)std::min<int64_t>(chunk, n_mat - first);
-        cudaError_t e = launch_project_simt(view, l.dtype, first, count, basis, sink, scratch, stream);
+        cudaError_t e;
+        {
+            TransformTimer timer(ctx, stream);
+            e = launch_project_simt(view, l.dtype, first, count, basis, sink, scratch, stream);
+        }
         if (e != cudaSuccess) return cuda_fail(ctx, e, "project_simt");
         e = launch_copy_back(view, l.dtype, first, count, n_keep, sink, scratch, stream);
         if (e != cudaSuccess) return cuda_fail(ctx, e, "copy_back");
+        ctx->kernels_launched += 2;
     }
     return FREQKV_OK;
 }
@@ -355,6 +411,13 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     gemm_release(&ctx->gemm);
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
+    for (int i = 0; i < 2; ++i)
+        if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    for (auto* list : {&ctx->pending, &ctx->spare})
+        for (auto& ev : *list) {
+            cudaEventDestroy(ev.first);
+            cudaEventDestroy(ev.second);
+        }
     cudaGetLastError();
     delete ctx;
     return FREQKV_OK;
@@ -496,7 +559,108 @@ freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* 
     const cudaError_t e =
         launch_append(view, layout->dtype, layout->batch, lens, n_new, new_k, new_v, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "append");
+    ctx->kernels_launched += (layout->batch + 127) / 128;
     for (int32_t b = 0; b < layout->batch; ++b) lens[b] += n_new;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout, void* k_host, void* v_host,
+                                   int32_t cache_len, int32_t kept_len, int32_t sink, void* cuda_stream,
+                                   int64_t* h2d_bytes, int64_t* d2h_bytes)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = freqkv_check_compress(layout, k_host, v_host, cache_len, kept_len, sink);
+    if (st != FREQKV_OK) return st;
+    if (h2d_bytes) *h2d_bytes = 0;
+    if (d2h_bytes) *d2h_bytes = 0;
+    const int32_t n_in = cache_len - sink;
+    if (n_in == 0 || kept_len == 0 || kept_len == n_in) return FREQKV_OK;
+    const freqkv_layout& l = *layout;
+    const int32_t variant = resolve(ctx, l, n_in, kept_len);
+    if (variant < 0) return FREQKV_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t elt = dtype_size(l.dtype);
+    const size_t bytes = (size_t)span_elements(l) * elt;
+    if (bytes > ctx->stage_bytes) {
+        FREQKV_CUDA(ctx, cudaDeviceSynchronize());
+        for (int i = 0; i < 2; ++i) {
+            if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+            ctx->stage[i] = nullptr;
+        }
+        ctx->stage_bytes = 0;
+        FREQKV_CUDA(ctx, cudaMalloc(&ctx->stage[0], bytes));
+        FREQKV_CUDA(ctx, cudaMalloc(&ctx->stage[1], bytes));
+        ctx->stage_bytes = bytes;
+    }
+    // One 2-D copy per (tensor, batch, layer): `kv_heads` runs of rows, one run per head.  Rows of
+    // a matrix are contiguous when stride_token == head_dim; padded rows are copied with their
+    // padding (same layout on both sides).
+    const size_t row_bytes = (size_t)l.stride_token * elt;
+    auto copy_rows = [&](bool to_device, int32_t row0, int32_t rows, int64_t* counter) -> cudaError_t {
+        const size_t width = rows == 0 ? 0 : (size_t)(rows - 1) * row_bytes + (size_t)l.head_dim * elt;
+        for (int t = 0; t < 2; ++t) {
+            char* host = static_cast<char*>(t ? v_host : k_host);
+            char* dev = static_cast<char*>(ctx->stage[t]);
+            for (int32_t b = 0; b < l.batch; ++b)
+                for (int32_t y = 0; y < l.layers; ++y) {
+                    const size_t off = ((size_t)b * l.stride_batch + (size_t)y * l.stride_layer + (size_t)row0 * l.stride_token) * elt;
+                    const size_t pitch = (size_t)l.stride_head * elt;
+                    cudaError_t e;
+                    if (l.kv_heads == 1 || pitch >= width)
+                        e = cudaMemcpy2DAsync(to_device ? dev + off : host + off, l.kv_heads == 1 ? width : pitch,
+                                              to_device ? host + off : dev + off, l.kv_heads == 1 ? width : pitch, width,
+                                              l.kv_heads, to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost,
+                                              stream);
+                    else
+                        e = cudaErrorInvalidValue;
+                    if (e != cudaSuccess) return e;
+                    if (counter) *counter += (int64_t)width * l.kv_heads;
+                }
+        }
+        return cudaSuccess;
+    };
+    // head stride below one matrix's rows (heads interleaved inside the token axis) is not
+    // something a 2-D copy can express
+    if (l.kv_heads > 1 && (size_t)l.stride_head * elt < (size_t)(n_in - 1) * row_bytes + (size_t)l.head_dim * elt)
+        return FREQKV_ERR_UNSUPPORTED;
+    cudaError_t e = copy_rows(true, sink, n_in, h2d_bytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "host->device copy");
+    st = compress_group(ctx, l, ctx->stage[0], ctx->stage[1], 0, l.batch, n_in, kept_len, sink, variant, stream);
+    if (st != FREQKV_OK) return st;
+    e = copy_rows(false, sink, kept_len, d2h_bytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "device->host copy");
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_set_timing(freqkv_ctx* ctx, int32_t enabled)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    ctx->timing = enabled != 0;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_get_timing(freqkv_ctx* ctx, int64_t* transform_launches, double* transform_ms,
+                                int64_t* kernels_launched)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    double ms = 0.0;
+    int64_t n = 0;
+    for (auto& ev : ctx->pending) {
+        FREQKV_CUDA(ctx, cudaEventSynchronize(ev.second));
+        float t = 0.f;
+        FREQKV_CUDA(ctx, cudaEventElapsedTime(&t, ev.first, ev.second));
+        ms += t;
+        ++n;
+        ctx->spare.push_back(ev);
+    }
+    ctx->pending.clear();
+    if (transform_launches) *transform_launches = n;
+    if (transform_ms) *transform_ms = ms;
+    if (kernels_launched) *kernels_launched = ctx->kernels_launched;
     return FREQKV_OK;
 }
 

@@ -6,12 +6,24 @@ namespace freqkv {
 
 struct GemmState {
     const char* last_error = nullptr;
+    int kernels_last_call = 0;
+    bool attr_set = false;
+    void* scratch = nullptr;  // output staging, [2][pairs][n_keep][128] bf16 per chunk
+    size_t scratch_bytes = 0;
+};
+
+// Called on the launching stream right before and right after the tensor-core kernel itself
+// (not the copy kernels around it), so that a caller can bracket it with events.
+struct LaunchHooks {
+    void (*before)(void* user, cudaStream_t stream) = nullptr;
+    void (*after)(void* user, cudaStream_t stream) = nullptr;
+    void* user = nullptr;
 };
 
 bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_keep);
 cudaError_t launch_gemm(GemmState* state, const CacheView& view, const freqkv_layout& layout, void* k, void* v,
                         int32_t batch0, int32_t batch_count, const Basis& basis, int32_t sink, int32_t* status_dev,
-                        int sm_count, cudaStream_t stream);
+                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 void gemm_release(GemmState* state);
 
 }  // namespace freqkv

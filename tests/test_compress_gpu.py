@@ -159,3 +159,46 @@ def test_ragged_batch_small(ctx):
                 assert parity.rel_l2(got, want) < 1e-2
                 assert torch.equal(t_out[b, 0, h, :4], t_in[b, 0, h, :4])
                 assert torch.equal(t_out[b, 0, h, 4 + kept[b]:], t_in[b, 0, h, 4 + kept[b]:])
+
+
+# ---- tensor-core projection (tcgen05 / TMEM / TMA), bf16 caches with head_dim 128
+@pytest.mark.parametrize("n_in,kept,sink", [(128, 64, 0), (256, 128, 4), (300, 150, 4), (700, 350, 4), (1000, 999, 1),
+                                            (1023, 511, 0), (1500, 100, 4), (64, 32, 2), (17, 5, 0)])
+def test_gemm_lengths(ctx, n_in, kept, sink):
+    w = small(cap=n_in + sink + 5, dtype=torch.bfloat16, sink=sink, outliers=2, Ly=1, H=2)
+    parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.GEMM)
+
+
+def test_gemm_batch_layers_heads_and_padding(ctx):
+    w = small(cap=333, dtype=torch.bfloat16, sink=4, outliers=2, B=2, Ly=3, H=2)
+    parity.check_compress(ctx, w, 330, 163, 4, fk.GEMM)
+    parity.check_compress(ctx, w, 333, 164, 4, fk.GEMM, row_pad=8)
+
+
+def test_gemm_many_tiles_more_than_sms(ctx):
+    """More output tiles than SMs, so every CTA runs several tiles through its pipeline."""
+    w = small(cap=600, dtype=torch.bfloat16, sink=4, outliers=2, B=1, Ly=8, H=16)
+    parity.check_compress(ctx, w, 600, 298, 4, fk.GEMM, sample=24)
+
+
+def test_config2_shape_gemm(ctx):
+    w = dataclasses.replace(synth.WORKLOADS["llama2_7b"], layers=2, kv_heads=8)
+    parity.check_compress(ctx, w, 4096, 2046, 4, fk.GEMM, sample=8)
+
+
+def test_config3_shape_gemm(ctx):
+    w = dataclasses.replace(synth.WORKLOADS["llama3_8b"], batch=2, layers=1, kv_heads=2)
+    parity.check_compress(ctx, w, 8192, 4094, 4, fk.GEMM, sample=4)
+
+
+def test_gemm_in_place_equals_fresh_copy(ctx):
+    """Running on a cache and on a clone of it gives bit-identical results (no dependence on
+    scheduling or on what the tiles of other matrices do)."""
+    w = small(cap=520, dtype=torch.bfloat16, sink=4, outliers=2, B=1, Ly=4, H=4)
+    k, v = synth.make_cache(w, "cuda")
+    k2, v2 = k.clone(), v.clone()
+    ctx.set_variant(fk.GEMM)
+    ctx.compress(k, v, 520, 258, 4)
+    ctx.compress(k2, v2, 520, 258, 4)
+    assert ctx.last_device_status() == fk.OK
+    assert torch.equal(k, k2) and torch.equal(v, v2)

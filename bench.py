@@ -206,7 +206,7 @@ def cpu_baseline(w, k, v, cache_len, kept, sink, budget_s=12.0):
     t0 = time.perf_counter()
     oracle.compress_matrix(x0, kept)
     one = time.perf_counter() - t0
-    count = int(max(2, min(64, budget_s / max(one, 1e-3))))
+    count = int(max(2, min(256, budget_s / max(one, 1e-3))))
     ids = torch.linspace(0, flat.shape[0] - 1, count).long().tolist()
     xs = [flat[i, sink:cache_len].to("cpu").to(torch.float64).numpy() for i in ids]
     t0 = time.perf_counter()
@@ -228,6 +228,7 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "gemm", "fdct", "simt"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="shrink the workload to this many layers (profiling only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank, local_rank, world = dist_env()
@@ -250,6 +251,10 @@ def main():
     n_gpus = world
 
     w = synth.WORKLOADS[args.workload]
+    if args.layers > 0:
+        import dataclasses
+
+        w = dataclasses.replace(w, layers=args.layers)
     cache_len, sink = w.capacity, w.sink
     kept = w.kept_len(cache_len)
     n_new = cache_len - sink - kept

@@ -145,6 +145,38 @@ freqkv_status freqkv_set_timing(freqkv_ctx* ctx, int32_t enabled);
 freqkv_status freqkv_get_timing(freqkv_ctx* ctx, int64_t* transform_launches, double* transform_ms,
                                 int64_t* kernels_launched);
 
+/* Compression for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of freqkv_compress, same definition, same result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not allowed or not safe -- inside a CUDA
+ * stream capture, under a lock that an allocation's implicit synchronisation could deadlock
+ * against, in a serving loop whose device-memory budget is frozen, or inside a host framework
+ * that owns all device memory.  freqkv_compress does not fit there: its context, its plan and
+ * its staging buffer all come from cudaMalloc.
+ *
+ * What it does: the CUDA-core (SIMT) projection of freqkv_compress with its two work areas --
+ * the fp32 projection basis and the staging area for compressed rows -- placed in fixed arrays
+ * inside the library image instead of allocated memory.  No context is needed; `k` and `v` are
+ * device pointers exactly as for freqkv_compress and the arrays of the device that owns them are
+ * used.  The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ * Limits (FREQKV_ERR_UNSUPPORTED beyond them, nothing enqueued): with n_in = cache_len - sink,
+ *   roundup(n_in, 64) * roundup(kept_len, 64) <= FREQKV_NOALLOC_MAX_BASIS_ELEMS   (1 Mi entries),
+ *   kept_len * head_dim * sizeof(element)     <= FREQKV_NOALLOC_STAGING_BYTES      (4 MiB);
+ * any number of matrices is accepted (they are processed in groups that fit the staging area).
+ * Cost: every GPU that loads the library holds the 8 MiB of arrays until the process exits.
+ *
+ * First call on a device: it looks up the device addresses of the arrays (once per device), so
+ * make the first call on each device before starting any stream capture.
+ * Sharing: all calls on a device share the arrays.  Calls on one stream are ordered and safe;
+ * calls whose kernels may overlap on the GPU (different streams, different threads) race on them
+ * and must be serialised by the caller.  Stale contents of earlier calls are never read: the
+ * part of the basis a call uses is rewritten by that call. */
+#define FREQKV_NOALLOC_MAX_BASIS_ELEMS (1u << 20)
+#define FREQKV_NOALLOC_STAGING_BYTES (4u << 20)
+freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
+                                      int32_t kept_len, int32_t sink, void* cuda_stream);
+
 /* Synchronise `cuda_stream`, then read and clear the device status word.  FREQKV_OK unless a
  * kernel's bounded wait (mbarrier / flag) ran out, in which case the affected output rows are
  * undefined and FREQKV_ERR_TIMEOUT is returned; the context stays usable. */

@@ -26,8 +26,10 @@ EXPORTS = [
     "freqkv_resolve_variant", "freqkv_plan", "freqkv_compress", "freqkv_compress_ragged",
     "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
-    "freqkv_set_timing", "freqkv_get_timing",
+    "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc",
 ]
+NOALLOC_MAX_BASIS_ELEMS = 1 << 20
+NOALLOC_STAGING_BYTES = 4 << 20
 
 
 class Layout(ctypes.Structure):
@@ -75,6 +77,7 @@ def lib() -> ctypes.CDLL:
                                            POINTER(c_int64), POINTER(c_int64)]
         L.freqkv_set_timing.argtypes = [c_void_p, c_int32]
         L.freqkv_get_timing.argtypes = [c_void_p, POINTER(c_int64), POINTER(ctypes.c_double), POINTER(c_int64)]
+        L.freqkv_compress_noalloc.argtypes = [LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -125,6 +128,21 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def compress_noalloc(k: torch.Tensor, v: torch.Tensor, cache_len: int, kept_len: int, sink: int, stream=None) -> int:
+    """``freqkv_compress_noalloc``: in-place compression without a context and without any
+    device allocation, for callers that cannot call cudaMalloc (stream capture, frozen memory
+    budgets).  Small shapes only: see the limits in ``include/freqkv.h``.  Returns the new
+    cache length; raises FreqKVError (ERR_UNSUPPORTED beyond the size limits)."""
+    lay = layout_of(k)
+    if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+        raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+    st = lib().freqkv_compress_noalloc(ctypes.byref(lay), k.data_ptr(), v.data_ptr(), cache_len, kept_len, sink,
+                                       _stream_ptr(stream))
+    if st != OK:
+        raise FreqKVError(st, f"freqkv_compress_noalloc: {status_string(st)}")
+    return sink + kept_len
 
 
 class Context:

@@ -202,3 +202,47 @@ def test_gemm_in_place_equals_fresh_copy(ctx):
     ctx.compress(k2, v2, 520, 258, 4)
     assert ctx.last_device_status() == fk.OK
     assert torch.equal(k, k2) and torch.equal(v, v2)
+
+
+# ---- fast-transform variant (power-of-two lengths), in place without scratch
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n_in,kept,sink", [(128, 64, 0), (256, 128, 4), (512, 256, 0), (1024, 128, 4), (2048, 16, 1),
+                                            (2048, 1024, 4), (4096, 2048, 0), (4096, 512, 4), (8192, 4096, 4)])
+def test_fdct_lengths(ctx, dtype, n_in, kept, sink):
+    w = small(cap=n_in + sink + 3, dtype=dtype, sink=sink, outliers=2 if dtype == torch.bfloat16 else 0, Ly=1, H=2)
+    parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.FDCT)
+
+
+def test_fdct_row_padding_batch_and_head_dim(ctx):
+    w = small(cap=520, dtype=torch.bfloat16, sink=4, outliers=2, B=2, Ly=2, H=2)
+    parity.check_compress(ctx, w, 516, 256, 4, fk.FDCT, row_pad=8)
+    w64 = small(cap=256, hd=64, dtype=torch.float32, sink=0, B=1, Ly=1, H=3)
+    parity.check_compress(ctx, w64, 256, 128, 0, fk.FDCT)
+
+
+def test_fdct_refuses_other_lengths(ctx):
+    k = torch.zeros(1, 1, 1, 600, 128, device="cuda", dtype=torch.bfloat16)
+    v = torch.zeros_like(k)
+    ctx.set_variant(fk.FDCT)
+    with pytest.raises(fk.FreqKVError) as e:
+        ctx.compress(k, v, 504, 250, 4)
+    assert e.value.status == fk.ERR_UNSUPPORTED
+    ctx.set_variant(fk.AUTO)
+
+
+def test_config2_pow2_shape_fdct(ctx):
+    w = dataclasses.replace(synth.WORKLOADS["llama2_7b_pow2"], layers=2, kv_heads=8)
+    parity.check_compress(ctx, w, 4096, 2048, 0, fk.FDCT, sample=8)
+
+
+def test_auto_picks_documented_variants(ctx):
+    ctx.set_variant(fk.AUTO)
+    bf = fk.layout_contiguous(fk.BF16, 1, 1, 1, 8192, 128)[1]
+    f32 = fk.layout_contiguous(fk.F32, 1, 1, 1, 8192, 128)[1]
+    assert ctx.resolve_variant(bf, 4096, 2048) == fk.GEMM
+    assert ctx.resolve_variant(fk.layout_contiguous(fk.BF16, 1, 1, 1, 8192, 64)[1], 4096, 2048) == fk.FDCT
+    assert ctx.resolve_variant(bf, 4092, 2046) == fk.GEMM
+    assert ctx.resolve_variant(bf, 8188, 4094) == fk.GEMM
+    assert ctx.resolve_variant(f32, 512, 256) == fk.FDCT
+    assert ctx.resolve_variant(f32, 500, 250) == fk.SIMT
+    assert ctx.resolve_variant(bf, 100, 50) == fk.SIMT

@@ -168,54 +168,67 @@ void free_bases(freqkv_ctx* ctx)
 {
     for (auto& kv : ctx->bases) {
         if (kv.second.f32) cudaFree(kv.second.f32);
-        if (kv.second.bf16) cudaFree(kv.second.bf16);
+        if (kv.second.fold) cudaFree(kv.second.fold);
     }
     ctx->bases.clear();
     ctx->basis_bytes = 0;
 }
 
-// Projection basis for (n_in, n_keep) holding at least the requested precisions.
-freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need_f32, bool need_bf16,
+// Projection basis for (n_in, n_keep) holding at least the requested forms: the full fp32 matrix
+// (CUDA-core path) and/or the folded bf16 pair Pe, Po (tensor-core path).
+freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need_f32, bool need_fold,
                         cudaStream_t stream, Basis* out)
 {
     const auto key = std::make_pair(n_in, n_keep);
     Basis b;
     auto it = ctx->bases.find(key);
     if (it != ctx->bases.end()) b = it->second;
-    const bool make_f32 = need_f32 && !b.f32, make_bf16 = need_bf16 && !b.bf16;
-    if (make_f32 || make_bf16) {
-        b.n_in = n_in;
-        b.n_keep = n_keep;
-        b.ld = (n_in + 63) / 64 * 64;
-        b.rows_pad = (n_keep + 63) / 64 * 64;
+    const bool make_f32 = need_f32 && !b.f32, make_fold = need_fold && !b.fold;
+    if (make_f32 || make_fold) {
+        auto shape = [&](Basis& x) {
+            x.n_in = n_in;
+            x.n_keep = n_keep;
+            x.ld = (n_in + 63) / 64 * 64;
+            x.rows_pad = (n_keep + 63) / 64 * 64;
+            x.fold_ld = ((n_in + 1) / 2 + 63) / 64 * 64;
+            x.fold_rows_pad = ((n_keep + 1) / 2 + 127) / 128 * 128;
+        };
+        shape(b);
         const size_t elems = (size_t)b.ld * b.rows_pad;
-        const size_t want = (make_f32 ? elems * 4 : 0) + (make_bf16 ? elems * 2 : 0);
+        const size_t fold_elems = (size_t)2 * b.fold_ld * b.fold_rows_pad;
+        const size_t want = (make_f32 ? elems * 4 : 0) + (make_fold ? fold_elems * 2 : 0);
         if (ctx->basis_bytes + want > kBasisBudgetBytes) {
             FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // bases may be in use by enqueued kernels
             free_bases(ctx);
             b = Basis();
-            b.n_in = n_in; b.n_keep = n_keep; b.ld = (n_in + 63) / 64 * 64; b.rows_pad = (n_keep + 63) / 64 * 64;
-            it = ctx->bases.end();
+            shape(b);
         }
         float* pf = nullptr;
         __nv_bfloat16* pb = nullptr;
         if (need_f32 && !b.f32) FREQKV_CUDA(ctx, cudaMalloc(&pf, elems * 4));
-        if (need_bf16 && !b.bf16) {
-            const cudaError_t e = cudaMalloc(&pb, elems * 2);
+        if (need_fold && !b.fold) {
+            const cudaError_t e = cudaMalloc(&pb, fold_elems * 2);
             if (e != cudaSuccess) {
                 if (pf) cudaFree(pf);
                 return cuda_fail(ctx, e, "cudaMalloc(basis)");
             }
         }
-        const cudaError_t e = launch_build_basis(pf, pb, n_in, n_keep, b.ld, b.rows_pad, stream);
+        cudaError_t e = cudaSuccess;
+        if (pf) {
+            e = launch_build_basis(pf, nullptr, n_in, n_keep, b.ld, b.rows_pad, stream);
+            ctx->kernels_launched += 1;
+        }
+        if (e == cudaSuccess && pb) {
+            e = launch_build_folded_basis(pb, n_in, n_keep, b.fold_ld, b.fold_rows_pad, stream);
+            ctx->kernels_launched += 1;
+        }
         if (e != cudaSuccess) {
             if (pf) cudaFree(pf);
             if (pb) cudaFree(pb);
             return cuda_fail(ctx, e, "build_basis");
         }
-        ctx->kernels_launched += 1;
         if (pf) { b.f32 = pf; ctx->basis_bytes += elems * 4; }
-        if (pb) { b.bf16 = pb; ctx->basis_bytes += elems * 2; }
+        if (pb) { b.fold = pb; ctx->basis_bytes += fold_elems * 2; }
         ctx->bases[key] = b;
     }
     *out = b;
@@ -310,8 +323,7 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
         hooks.user = &timer;
         hooks.before = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->begin(); };
         hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
-        const cudaError_t e = launch_gemm(&ctx->gemm, view, l, k, v, batch0, batch_count, basis, sink, ctx->status_dev,
-                                          ctx->sm_count, hooks, stream);
+        const cudaError_t e = launch_gemm(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
         if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
         ctx->kernels_launched += ctx->gemm.kernels_last_call;
         return FREQKV_OK;

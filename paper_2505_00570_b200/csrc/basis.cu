@@ -43,7 +43,47 @@ __global__ void build_basis_kernel(float* __restrict__ p_f32, __nv_bfloat16* __r
     }
 }
 
+// Folded basis for the tensor-core path.  The cosines of the DCT are symmetric or antisymmetric
+// under n -> N-1-n and m -> L-1-m according to the parity of the frequency index t, so
+// P[m][N-1-n] = Pe[m][n] - Po[m][n] and P[L-1-m][n] = Pe[m][n] - Po[m][n], where Pe (Po) is the part
+// of the sum over even (odd) t:  Pe = (P[m][n] + P[m][N-1-n]) / 2,  Po = (P[m][n] - P[m][N-1-n]) / 2.
+// Only m < ceil(L/2), n < ceil(N/2) are stored: plane 0 = Pe, plane 1 = Po, each rows_pad x ld,
+// zero padded.  For odd N the middle column of Po is zero and that of Pe is P itself, for odd L the
+// middle row of Po is zero: the formulas above give exactly that.
+__global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32_t n_in, int32_t n_keep, int32_t ld,
+                                          int32_t rows_pad)
+{
+    const int64_t plane = (int64_t)rows_pad * ld;
+    const int64_t N = n_in, L = n_keep, LN4 = 4 * L * N;
+    const int64_t Nh = (N + 1) / 2, Lh = (L + 1) / 2;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = i / ld, n = i % ld;
+        double pe = 0.0, po = 0.0;
+        if (m < Lh && n < Nh) {
+            const int64_t u = (2 * m + 1) * N, w = (2 * n + 1) * L, wr = (2 * (N - 1 - n) + 1) * L;
+            const double a = (dirichlet(u + w, L, LN4) + dirichlet(u - w, L, LN4)) / (double)(2 * N);
+            const double b = (dirichlet(u + wr, L, LN4) + dirichlet(u - wr, L, LN4)) / (double)(2 * N);
+            pe = 0.5 * (a + b);
+            po = 0.5 * (a - b);
+        }
+        out[i] = __double2bfloat16(pe);
+        out[plane + i] = __double2bfloat16(po);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
+                                      cudaStream_t stream)
+{
+    const int64_t total = (int64_t)rows_pad * ld;
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks < 1) blocks = 1;
+    build_folded_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(out, n_in, n_keep, ld, rows_pad);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
                                int32_t rows_pad, cudaStream_t stream)

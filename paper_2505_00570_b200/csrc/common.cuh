@@ -36,9 +36,12 @@ __host__ __device__ inline void* tensor_base(const CacheView& v, int32_t tensor)
 // Projection basis of one (n_in, n_keep) pair: P[m][n], row-major with leading dimension ld,
 // rows padded to rows_pad and columns to ld with zeros.
 struct Basis {
-    float* f32 = nullptr;          // SIMT path
-    __nv_bfloat16* bf16 = nullptr; // tensor-core path
+    float* f32 = nullptr;  // SIMT path
     int32_t n_in = 0, n_keep = 0, ld = 0, rows_pad = 0;
+    // Tensor-core path: the even-frequency and odd-frequency parts Pe, Po of P restricted to
+    // m < ceil(n_keep/2), n < ceil(n_in/2), bf16, two planes of fold_rows_pad x fold_ld (see basis.cu).
+    __nv_bfloat16* fold = nullptr;
+    int32_t fold_ld = 0, fold_rows_pad = 0;
 };
 
 // ---- kernel launchers (each returns the cudaError_t of its launch) ----
@@ -46,6 +49,10 @@ struct Basis {
 // P[m][n] for m < n_keep, n < n_in from the closed form; zero padding elsewhere.
 cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
                                int32_t rows_pad, cudaStream_t stream);
+
+// Pe and Po of the folded basis (two planes of rows_pad x ld), zero padding elsewhere.
+cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
+                                      cudaStream_t stream);
 
 // scratch[i - first][m][c] = sum_n P[m][n] * X_i[sink + n][c] for matrices first .. first+count-1.
 cudaError_t launch_project_simt(const CacheView& view, int32_t dtype, int32_t first, int32_t count, const Basis& basis,

@@ -2,23 +2,31 @@
 // of Appendix A folded into the basis P, see basis.cu) on the 5th-generation tensor cores of
 // sm_100a: tcgen05.mma with accumulators in tensor memory, operands staged by TMA.
 //
-// Shape of the problem.  P is L x N (bf16, row-major: the contraction axis is contiguous, a
-// "K-major" A operand) and is shared by every matrix.  X_i is N x 128 per (batch, layer,
-// kv_head) and tensor (K or V), with the 128 channels contiguous: an "MN-major" B operand.  The
-// K matrix and the V matrix of the same (batch, layer, kv_head) sit side by side in one
-// 256-column B tile, so K and V are compressed by the same launch and the same instructions.
+// Symmetry fold.  The DCT cosines are even or odd under n -> N-1-n (and m -> L-1-m) according to
+// the parity of the frequency t, so with P = Pe + Po split into its even-t and odd-t parts
+//     u_n = x_n + x_{N-1-n},   v_n = x_n - x_{N-1-n}            (n < ceil(N/2))
+//     s_m = sum_n Pe[m][n] u_n,   d_m = sum_n Po[m][n] v_n      (m < ceil(L/2))
+//     y_m = s_m + d_m,   y_{L-1-m} = s_m - d_m
+// which is the same linear map with half the multiply-adds.  (For odd N the middle row enters u
+// once and v as zero; for odd L the middle output row has d = 0 and is written once.)
 //
-// One CTA per SM, persistent over output tiles of 256 rows x 256 columns:
-//   warp 0      TMA producer: per 64-token slice of the contraction, 2 boxes of P (128 rows x 64)
-//               and 4 boxes of X (64 tokens x 64 channels; K low/high, V low/high), 128-byte
-//               swizzled, into a 3-stage ring of 64 KB stages;
-//   warp 1      MMA issuer: per stage 4 (k = 16) x 2 (row halves) tcgen05.mma of 128 x 256 x 16
-//               into 2 x 256 fp32 columns of tensor memory (all 512 columns of the SM);
-//   warps 2-9   epilogue: tcgen05.ld, round to bf16 (nearest even), 16-byte global stores.
-//
-// Every output row of a matrix depends on every input row of the same matrix and the output
-// rows overwrite input rows, so tiles write to a scratch buffer; a copy kernel moves the rows
-// into the cache when the launch is over.
+// Two kernels per call:
+//   fold_kernel         reads every non-sink cache row once and writes U and V (bf16) to a scratch
+//                       buffer, one plane of ceil(N/2) x 128 per (matrix, u|v); HBM-bound.
+//   freqkv_gemm_kernel  one CTA per SM, persistent over output tiles of 128 folded rows x 256
+//                       columns (the K matrix and the V matrix of one (batch, layer, kv_head) side
+//                       by side, so K and V share every instruction).  Per tile it first accumulates
+//                       S = Pe U, then D = Po V, in the two halves of tensor memory:
+//     warp 0      TMA producer: per 64-row slice of the contraction one box of Pe or Po (128 x 64)
+//                 and 4 boxes of U or V (64 rows x 64 channels), 128-byte swizzled, into a ring
+//                 of 4 stages of 48 KB;
+//     warp 1      MMA issuer: 4 tcgen05.mma (128 x 256 x 16) per stage;
+//     warps 2-9   epilogue: when S is complete they park it in registers (which frees that half
+//                 of tensor memory for the next tile while D is still accumulating); when D is
+//                 complete they form s + d and s - d, round to bf16 (nearest even) and store rows
+//                 m and L-1-m straight into the cache.  Both steps overlap the MMAs of the
+//                 neighbouring phases, so the tensor pipe never waits for the epilogue.
+// The kernel reads only the scratch planes and the basis, so writing the cache in place is safe.
 //
 // Every wait on an mbarrier is bounded in time: a wait that runs out sets a bit in the status
 // word, raises a CTA-wide abort flag that ends every other role's loop, the producer drains
@@ -33,15 +41,13 @@
 namespace freqkv {
 namespace {
 
-constexpr int BM = 256;        // output rows per tile (two UMMA row halves of 128)
-constexpr int BN = 256;        // output columns per tile: K channels 0..127 | V channels 0..127
-constexpr int BK = 64;         // contraction slice per stage (tokens)
-constexpr int STAGES = 3;
-constexpr int A_HALF_BYTES = 128 * BK * 2;         // 16 KB: 128 rows x 64 bf16, 128 B per row
-constexpr int A_BYTES = 2 * A_HALF_BYTES;          // 32 KB
-constexpr int B_CHUNK_BYTES = BK * 128;            // 8 KB: 64 tokens x 64 channels
+constexpr int BM = 128;        // folded output rows per tile (one UMMA of M = 128 per accumulator); 256 columns: K | V
+constexpr int BK = 64;         // contraction slice per stage (folded rows)
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;               // 16 KB: 128 rows x 64 bf16, 128 B per row
+constexpr int B_CHUNK_BYTES = BK * 128;            // 8 KB: 64 rows x 64 channels
 constexpr int B_BYTES = 4 * B_CHUNK_BYTES;         // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 64 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 48 KB
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int NUM_THREADS = 320;                   // 10 warps
 constexpr int EPI_WARPS = 8;
@@ -51,11 +57,12 @@ constexpr uint32_t ERR_FULL_WAIT = 1u, ERR_EMPTY_WAIT = 2u, ERR_ACC_FULL_WAIT = 
                    ERR_DRAIN_WAIT = 16u;
 
 struct GemmParams {
-    int32_t n_in, n_keep;       // N, L
+    int32_t n_keep;             // L
+    int32_t rows_half;          // ceil(L / 2): folded output rows
+    int32_t basis_rows_pad;     // row offset of the Po plane inside the basis tensor map
     int32_t pair0, pair_count;  // (batch, layer, kv_head) triples covered by this launch
-    int32_t layers, kv_heads;
     int32_t m_tiles, k_steps;
-    __nv_bfloat16* scratch;     // [2][pair_count][n_keep][128]
+    int32_t sink;
     int32_t* status;
 };
 
@@ -125,12 +132,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t c0, int32_t c1,
-                                            int32_t c2, int32_t c3, int32_t c4)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t c0, int32_t c1,
+                                            int32_t c2)
 {
     asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 
@@ -166,29 +173,93 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+// 32 lanes x 32 consecutive columns of tensor memory into registers r[OFF .. OFF+31].
+template <int OFF, int NREG>
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[NREG])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "=r"(r[OFF + 0]), "=r"(r[OFF + 1]), "=r"(r[OFF + 2]), "=r"(r[OFF + 3]), "=r"(r[OFF + 4]), "=r"(r[OFF + 5]),
+          "=r"(r[OFF + 6]), "=r"(r[OFF + 7]), "=r"(r[OFF + 8]), "=r"(r[OFF + 9]), "=r"(r[OFF + 10]), "=r"(r[OFF + 11]),
+          "=r"(r[OFF + 12]), "=r"(r[OFF + 13]), "=r"(r[OFF + 14]), "=r"(r[OFF + 15]), "=r"(r[OFF + 16]),
+          "=r"(r[OFF + 17]), "=r"(r[OFF + 18]), "=r"(r[OFF + 19]), "=r"(r[OFF + 20]), "=r"(r[OFF + 21]),
+          "=r"(r[OFF + 22]), "=r"(r[OFF + 23]), "=r"(r[OFF + 24]), "=r"(r[OFF + 25]), "=r"(r[OFF + 26]),
+          "=r"(r[OFF + 27]), "=r"(r[OFF + 28]), "=r"(r[OFF + 29]), "=r"(r[OFF + 30]), "=r"(r[OFF + 31])
         : "r"(taddr)
         : "memory");
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits)
+// 32 lanes x 16 consecutive columns.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 {
-    const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(lo_bits), __uint_as_float(hi_bits));
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// ---- fold: U = X + reversed X, V = X - reversed X, one 16-byte vector (8 channels) per item ----
+
+__device__ __forceinline__ void fold8(const uint4& a, const uint4& b, uint4* u, uint4* v)
+{
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    uint32_t uw[4], vw[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float a0 = __uint_as_float(aw[i] << 16), a1 = __uint_as_float(aw[i] & 0xffff0000u);
+        const float b0 = __uint_as_float(bw[i] << 16), b1 = __uint_as_float(bw[i] & 0xffff0000u);
+        uw[i] = pack_bf16(a0 + b0, a1 + b1);
+        vw[i] = pack_bf16(a0 - b0, a1 - b1);
+    }
+    *u = make_uint4(uw[0], uw[1], uw[2], uw[3]);
+    *v = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+}
+
+// scratch planes: ((pair_local * 2 + tensor) * 2 + (0 = U, 1 = V)) of n_half rows x 128 channels.
+__global__ void __launch_bounds__(256) fold_kernel(CacheView view, int32_t pair0, int32_t pair_count, int32_t n_in,
+                                                   int32_t n_half, int32_t sink, uint4* __restrict__ scratch)
+{
+    const int64_t per_mat = (int64_t)n_half * 16;
+    const int64_t total = (int64_t)pair_count * 2 * per_mat;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int32_t vcol = (int32_t)(i & 15);
+        const int64_t row = i >> 4;
+        const int32_t n = (int32_t)(row % n_half);
+        const int32_t pt = (int32_t)(row / n_half);  // pair_local * 2 + tensor
+        const int32_t tensor = pt & 1;
+        const char* x = static_cast<const char*>(tensor_base(view, tensor)) +
+                        (matrix_offset(view, pair0 + (pt >> 1)) + (int64_t)sink * view.stride_token) * 2;
+        const int32_t nr = n_in - 1 - n;
+        const uint4 a = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * view.stride_token * 2) + vcol);
+        uint4 u, v;
+        if (nr != n) {
+            const uint4 b = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)nr * view.stride_token * 2) + vcol);
+            fold8(a, b, &u, &v);
+        } else {  // middle row of an odd-length signal
+            u = a;
+            v = make_uint4(0u, 0u, 0u, 0u);
+        }
+        uint4* pu = scratch + ((int64_t)pt * 2 * n_half + n) * 16 + vcol;
+        pu[0] = u;
+        pu[per_mat] = v;
+    }
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const GemmParams prm)
+freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_x,
+                   const CacheView view, const GemmParams prm)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -196,11 +267,12 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     uint8_t* aligned = smem_raw + (base - raw);
     uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
     const uint32_t bar0 = base + STAGES * STAGE_BYTES;
-    // barrier slots: full[0..S), empty[S..2S), acc_full (2S), acc_empty (2S+1)
+    // barrier slots: full[0..S), empty[S..2S), then s_full, s_empty, d_full, d_empty
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-    const uint32_t acc_full_bar = bar0 + 8u * (2 * STAGES), acc_empty_bar = bar0 + 8u * (2 * STAGES + 1);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+    auto acc_full_bar = [&](int eo) { return bar0 + 8u * (2 * STAGES + 2 * eo); };
+    auto acc_empty_bar = [&](int eo) { return bar0 + 8u * (2 * STAGES + 2 * eo + 1); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -211,13 +283,15 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
-        mbar_init(acc_full_bar, 1);
-        mbar_init(acc_empty_bar, EPI_WARPS);
+        for (int eo = 0; eo < 2; ++eo) {
+            mbar_init(acc_full_bar(eo), 1);
+            mbar_init(acc_empty_bar(eo), EPI_WARPS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {  // tensor memory: all 512 columns
+    if (warp == 1) {  // tensor memory: all 512 columns (S in 0..255, D in 256..511)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
@@ -232,26 +306,26 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             uint32_t it = 0;  // global slice counter: stage = it % STAGES, phase = it / STAGES
             bool alive = true;
             for (int32_t tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x) {
-                const int32_t pair = prm.pair0 + tile / prm.m_tiles, mt = tile % prm.m_tiles;
-                const int32_t h = pair % prm.kv_heads, l = (pair / prm.kv_heads) % prm.layers,
-                              b = pair / (prm.kv_heads * prm.layers);
-                for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
-                    const int s = it % STAGES;
-                    if (it >= STAGES &&
-                        !mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag, prm.status, ERR_EMPTY_WAIT)) {
-                        alive = false;
-                        break;
+                const int32_t pair_local = tile / prm.m_tiles, mt = tile % prm.m_tiles;
+                for (int eo = 0; eo < 2 && alive; ++eo) {
+                    for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
+                        const int s = it % STAGES;
+                        if (it >= STAGES &&
+                            !mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag, prm.status, ERR_EMPTY_WAIT)) {
+                            alive = false;
+                            break;
+                        }
+                        const uint32_t stage = base + s * STAGE_BYTES;
+                        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+                        const int32_t k0 = ks * BK;
+                        tma_load_2d(stage, &map_p, full_bar(s), k0, eo * prm.basis_rows_pad + mt * BM);
+                        const uint32_t bs = stage + A_BYTES;
+                        const int32_t plane_k = (pair_local * 2 + 0) * 2 + eo, plane_v = (pair_local * 2 + 1) * 2 + eo;
+                        tma_load_3d(bs + 0 * B_CHUNK_BYTES, &map_x, full_bar(s), 0, k0, plane_k);
+                        tma_load_3d(bs + 1 * B_CHUNK_BYTES, &map_x, full_bar(s), 64, k0, plane_k);
+                        tma_load_3d(bs + 2 * B_CHUNK_BYTES, &map_x, full_bar(s), 0, k0, plane_v);
+                        tma_load_3d(bs + 3 * B_CHUNK_BYTES, &map_x, full_bar(s), 64, k0, plane_v);
                     }
-                    const uint32_t stage = base + s * STAGE_BYTES;
-                    mbar_expect_tx(full_bar(s), STAGE_BYTES);
-                    const int32_t k0 = ks * BK;
-                    tma_load_2d(stage, &map_p, full_bar(s), k0, mt * BM);
-                    tma_load_2d(stage + A_HALF_BYTES, &map_p, full_bar(s), k0, mt * BM + 128);
-                    const uint32_t bs = stage + A_BYTES;
-                    tma_load_5d(bs + 0 * B_CHUNK_BYTES, &map_k, full_bar(s), 0, k0, h, l, b);
-                    tma_load_5d(bs + 1 * B_CHUNK_BYTES, &map_k, full_bar(s), 64, k0, h, l, b);
-                    tma_load_5d(bs + 2 * B_CHUNK_BYTES, &map_v, full_bar(s), 0, k0, h, l, b);
-                    tma_load_5d(bs + 3 * B_CHUNK_BYTES, &map_v, full_bar(s), 64, k0, h, l, b);
                 }
             }
             if (*abort_flag) {
@@ -269,69 +343,91 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             uint32_t it = 0, tile_no = 0;
             bool alive = true;
             for (int32_t tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++tile_no) {
-                if (tile_no > 0) {  // accumulators must have been drained by the epilogue
-                    if (!mbar_wait(acc_empty_bar, (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT)) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                }
-                for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
-                    const int s = it % STAGES;
-                    if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, prm.status, ERR_FULL_WAIT)) {
-                        alive = false;
-                        break;
-                    }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a0 = base + s * STAGE_BYTES, b0 = a0 + A_BYTES;
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) {
-                        // B: 4 chunks of 64 channels 8 KB apart (leading offset), 8-token groups 1 KB apart
-                        const uint64_t bd = smem_desc(b0 + kk * 2048, B_CHUNK_BYTES, 1024);
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            // A: 128 rows, 8-row groups 1 KB apart; 16 k-elements = 32 bytes inside the swizzled row
-                            const uint64_t ad = smem_desc(a0 + half * A_HALF_BYTES + kk * 32, 16, 1024);
-                            umma_bf16(tmem_base + half * 256, ad, bd, (ks | kk) != 0);
+                for (int eo = 0; eo < 2 && alive; ++eo) {
+                    if (tile_no > 0) {  // this accumulator must have been read by the epilogue of the last tile
+                        if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT)) {
+                            alive = false;
+                            break;
                         }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     }
-                    umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+                    for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
+                        const int s = it % STAGES;
+                        if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, prm.status, ERR_FULL_WAIT)) {
+                            alive = false;
+                            break;
+                        }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t a0 = base + s * STAGE_BYTES, b0 = a0 + A_BYTES;
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            // A: 128 rows, 8-row groups 1 KB apart; 16 k-elements = 32 bytes inside the swizzled row
+                            const uint64_t ad = smem_desc(a0 + kk * 32, 16, 1024);
+                            // B: 4 chunks of 64 channels 8 KB apart (leading offset), 8-row groups 1 KB apart
+                            const uint64_t bd = smem_desc(b0 + kk * 2048, B_CHUNK_BYTES, 1024);
+                            umma_bf16(tmem_base + eo * 256, ad, bd, (ks | kk) != 0);
+                        }
+                        umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+                    }
+                    if (alive) umma_commit(acc_full_bar(eo));
                 }
-                if (alive) umma_commit(acc_full_bar);
             }
         }
     } else {
         // ---------------- epilogue ----------------
-        const int ew = warp - 2, quarter = warp % 4, half = ew / 4;
+        const int ew = warp - 2, quarter = warp % 4, tensor = ew / 4;  // tensor: 0 = K columns, 1 = V columns
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tensor * 128;
         uint32_t tile_no = 0;
         for (int32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_no) {
-            if (!mbar_wait(acc_full_bar, tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
+            // S = Pe U: park this thread's row (128 columns) in registers, release that half
+            if (!mbar_wait(acc_full_bar(0), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            uint32_t s[128];
+            tmem_ld32<0>(lane_addr + 0, s);
+            tmem_ld32<32>(lane_addr + 32, s);
+            tmem_ld32<64>(lane_addr + 64, s);
+            tmem_ld32<96>(lane_addr + 96, s);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(0));
+
+            // D = Po V: combine and store rows m and L-1-m
+            if (!mbar_wait(acc_full_bar(1), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int32_t pair_local = tile / prm.m_tiles, mt = tile % prm.m_tiles;
-            const int32_t m = mt * BM + half * 128 + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * 256;
-#pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
-                uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (m < prm.n_keep) {
-                    const int tensor = c / 4;
-                    __nv_bfloat16* out = prm.scratch +
-                                         (((int64_t)tensor * prm.pair_count + pair_local) * prm.n_keep + m) * 128 +
-                                         (c % 4) * 32;
-                    uint4* o4 = reinterpret_cast<uint4*>(out);
+            const int32_t m = mt * BM + quarter * 32 + lane;
+            const int32_t mr = prm.n_keep - 1 - m;
+            const bool row_ok = m < prm.rows_half;
+            __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
+                                 matrix_offset(view, prm.pair0 + pair_local) + (int64_t)prm.sink * view.stride_token;
+            uint4* out_p = reinterpret_cast<uint4*>(mat + (int64_t)m * view.stride_token);
+            uint4* out_m = reinterpret_cast<uint4*>(mat + (int64_t)mr * view.stride_token);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 v;
-                        v.x = pack_bf16(r[8 * q + 0], r[8 * q + 1]);
-                        v.y = pack_bf16(r[8 * q + 2], r[8 * q + 3]);
-                        v.z = pack_bf16(r[8 * q + 4], r[8 * q + 5]);
-                        v.w = pack_bf16(r[8 * q + 6], r[8 * q + 7]);
-                        o4[q] = v;
+            for (int c = 0; c < 8; ++c) {
+                uint32_t d[16];
+                tmem_ld16(lane_addr + 256 + c * 16, d);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row_ok) {
+                    uint32_t p[8], q[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float s0 = __uint_as_float(s[c * 16 + 2 * j]), s1 = __uint_as_float(s[c * 16 + 2 * j + 1]);
+                        const float d0 = __uint_as_float(d[2 * j]), d1 = __uint_as_float(d[2 * j + 1]);
+                        p[j] = pack_bf16(s0 + d0, s1 + d1);
+                        q[j] = pack_bf16(s0 - d0, s1 - d1);
+                    }
+                    out_p[2 * c] = make_uint4(p[0], p[1], p[2], p[3]);
+                    out_p[2 * c + 1] = make_uint4(p[4], p[5], p[6], p[7]);
+                    if (mr != m) {
+                        out_m[2 * c] = make_uint4(q[0], q[1], q[2], q[3]);
+                        out_m[2 * c + 1] = make_uint4(q[4], q[5], q[6], q[7]);
                     }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar);
+            if (lane == 0) mbar_arrive(acc_empty_bar(1));
         }
     }
 
@@ -364,37 +460,31 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
+// Pe stacked over Po: a 2-D tensor of 2 * fold_rows_pad rows x fold_ld columns.
 bool encode_basis_map(CUtensorMap* map, const Basis& basis)
 {
-    const cuuint64_t dims[2] = {(cuuint64_t)basis.ld, (cuuint64_t)basis.rows_pad};
-    const cuuint64_t strides[1] = {(cuuint64_t)basis.ld * 2};
-    const cuuint32_t box[2] = {BK, 128};
+    const cuuint64_t dims[2] = {(cuuint64_t)basis.fold_ld, (cuuint64_t)2 * basis.fold_rows_pad};
+    const cuuint64_t strides[1] = {(cuuint64_t)basis.fold_ld * 2};
+    const cuuint32_t box[2] = {BK, BM};
     const cuuint32_t elem[2] = {1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, basis.bf16, dims, strides, box, elem,
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, basis.fold, dims, strides, box, elem,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The non-sink rows of one cache tensor as a 5-D tensor (channel, token, kv_head, layer, batch).
-bool encode_cache_map(CUtensorMap* map, const freqkv_layout& l, void* base, int32_t batch0, int32_t batch_count,
-                      int32_t n_in, int32_t sink)
+// The scratch planes as a 3-D tensor (channel, folded row, plane); rows past n_half read as zero.
+bool encode_scratch_map(CUtensorMap* map, void* scratch, int32_t n_half, int32_t planes)
 {
-    char* p = static_cast<char*>(base) + ((int64_t)batch0 * l.stride_batch + (int64_t)sink * l.stride_token) * 2;
-    const cuuint64_t dims[5] = {(cuuint64_t)l.head_dim, (cuuint64_t)n_in, (cuuint64_t)l.kv_heads, (cuuint64_t)l.layers,
-                                (cuuint64_t)batch_count};
-    // an axis of extent 1 is never stepped; give it a harmless stride
-    const cuuint64_t row = (cuuint64_t)l.stride_token * 2;
-    const cuuint64_t strides[4] = {row, l.kv_heads > 1 ? (cuuint64_t)l.stride_head * 2 : row,
-                                   l.layers > 1 ? (cuuint64_t)l.stride_layer * 2 : row,
-                                   batch_count > 1 ? (cuuint64_t)l.stride_batch * 2 : row};
-    const cuuint32_t box[5] = {64, BK, 1, 1, 1};
-    const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
-    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, p, dims, strides, box, elem,
+    const cuuint64_t dims[3] = {128, (cuuint64_t)n_half, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {256, (cuuint64_t)n_half * 256};
+    const cuuint32_t box[3] = {64, BK, 1};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, scratch, dims, strides, box, elem,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t kGemmScratchBytes = size_t(1) << 30;
+constexpr size_t kFoldScratchBytes = size_t(2304) << 20;  // one 7B-shaped cache of 4096 tokens fits in one pass
 
 }  // namespace
 
@@ -403,8 +493,7 @@ bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_kee
     return dtype == FREQKV_BF16 && head_dim == 128 && n_in >= 1 && n_keep >= 1 && n_keep <= n_in;
 }
 
-cudaError_t launch_gemm(GemmState* state, const CacheView& view, const freqkv_layout& layout, void* k, void* v,
-                        int32_t batch0, int32_t batch_count, const Basis& basis, int32_t sink, int32_t* status_dev,
+cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
                         int sm_count, const LaunchHooks& hooks, cudaStream_t stream)
 {
     state->kernels_last_call = 0;
@@ -421,17 +510,10 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const freqkv_la
         }
         state->attr_set = true;
     }
-    CUtensorMap map_p, map_k, map_v;
-    if (!encode_basis_map(&map_p, basis) ||
-        !encode_cache_map(&map_k, layout, k, batch0, batch_count, basis.n_in, sink) ||
-        !encode_cache_map(&map_v, layout, v, batch0, batch_count, basis.n_in, sink)) {
-        state->last_error = "tensor map encoding rejected this layout";
-        return cudaErrorInvalidValue;
-    }
-
+    const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
     const int32_t pairs = view.mats_per_tensor;
-    const size_t per_pair = (size_t)2 * basis.n_keep * 128 * 2;
-    int32_t chunk = (int32_t)std::max<size_t>(1, std::min<size_t>(kGemmScratchBytes / per_pair, (size_t)pairs));
+    const size_t per_pair = (size_t)4 * n_half * 128 * 2;  // K and V, U and V planes
+    const int32_t chunk = (int32_t)std::max<size_t>(1, std::min<size_t>(kFoldScratchBytes / per_pair, (size_t)pairs));
     if ((size_t)chunk * per_pair > state->scratch_bytes) {
         if (state->scratch) {
             cudaError_t e = cudaDeviceSynchronize();
@@ -442,45 +524,54 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const freqkv_la
         }
         const cudaError_t e = cudaMalloc(&state->scratch, (size_t)chunk * per_pair);
         if (e != cudaSuccess) {
-            state->last_error = "cudaMalloc(gemm scratch)";
+            state->last_error = "cudaMalloc(fold scratch)";
             return e;
         }
         state->scratch_bytes = (size_t)chunk * per_pair;
     }
+    CUtensorMap map_p;
+    if (!encode_basis_map(&map_p, basis)) {
+        state->last_error = "tensor map encoding rejected the basis";
+        return cudaErrorInvalidValue;
+    }
 
     for (int32_t p0 = 0; p0 < pairs; p0 += chunk) {
         const int32_t count = std::min(chunk, pairs - p0);
+        CUtensorMap map_x;
+        if (!encode_scratch_map(&map_x, state->scratch, n_half, count * 4)) {
+            state->last_error = "tensor map encoding rejected the scratch planes";
+            return cudaErrorInvalidValue;
+        }
+        const int64_t items = (int64_t)count * 2 * n_half * 16;
+        const unsigned fold_grid = (unsigned)std::min<int64_t>((items + 255) / 256, (int64_t)sm_count * 16);
+        fold_kernel<<<fold_grid, 256, 0, stream>>>(view, p0, count, basis.n_in, n_half, sink,
+                                                  static_cast<uint4*>(state->scratch));
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) {
+            state->last_error = "fold_kernel launch";
+            return e;
+        }
         GemmParams prm;
-        prm.n_in = basis.n_in;
         prm.n_keep = basis.n_keep;
+        prm.rows_half = rows_half;
+        prm.basis_rows_pad = basis.fold_rows_pad;
         prm.pair0 = p0;
         prm.pair_count = count;
-        prm.layers = view.layers;
-        prm.kv_heads = view.kv_heads;
-        prm.m_tiles = (basis.n_keep + BM - 1) / BM;
-        prm.k_steps = (basis.n_in + BK - 1) / BK;
-        prm.scratch = static_cast<__nv_bfloat16*>(state->scratch);
+        prm.m_tiles = (rows_half + BM - 1) / BM;
+        prm.k_steps = (n_half + BK - 1) / BK;
+        prm.sink = sink;
         prm.status = status_dev;
         const int32_t tiles = count * prm.m_tiles;
         const int grid = std::min<int32_t>(tiles, sm_count);
         if (hooks.before) hooks.before(hooks.user, stream);
-        freqkv_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_p, map_k, map_v, prm);
-        cudaError_t e = cudaGetLastError();
+        freqkv_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_p, map_x, view, prm);
+        e = cudaGetLastError();
         if (hooks.after) hooks.after(hooks.user, stream);
         if (e != cudaSuccess) {
             state->last_error = "freqkv_gemm_kernel launch";
             return e;
         }
-        const __nv_bfloat16* sk = prm.scratch;
-        const __nv_bfloat16* sv = prm.scratch + (size_t)count * basis.n_keep * 128;
-        e = launch_copy_back(view, FREQKV_BF16, p0, count, basis.n_keep, sink, sk, stream);
-        if (e == cudaSuccess)
-            e = launch_copy_back(view, FREQKV_BF16, view.mats_per_tensor + p0, count, basis.n_keep, sink, sv, stream);
-        if (e != cudaSuccess) {
-            state->last_error = "copy_back launch";
-            return e;
-        }
-        state->kernels_last_call += 3;
+        state->kernels_last_call += 2;
     }
     return cudaSuccess;
 }

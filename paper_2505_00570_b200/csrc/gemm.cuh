@@ -8,7 +8,7 @@ struct GemmState {
     const char* last_error = nullptr;
     int kernels_last_call = 0;
     bool attr_set = false;
-    void* scratch = nullptr;  // output staging, [2][pairs][n_keep][128] bf16 per chunk
+    void* scratch = nullptr;  // folded inputs U, V: [pairs][K|V][U|V][ceil(n_in/2)][128] bf16 per pass
     size_t scratch_bytes = 0;
 };
 
@@ -21,8 +21,7 @@ struct LaunchHooks {
 };
 
 bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_keep);
-cudaError_t launch_gemm(GemmState* state, const CacheView& view, const freqkv_layout& layout, void* k, void* v,
-                        int32_t batch0, int32_t batch_count, const Basis& basis, int32_t sink, int32_t* status_dev,
+cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
                         int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 void gemm_release(GemmState* state);
 

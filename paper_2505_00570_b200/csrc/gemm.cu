@@ -226,35 +226,63 @@ __device__ __forceinline__ void fold8(const uint4& a, const uint4& b, uint4* u, 
     *v = make_uint4(vw[0], vw[1], vw[2], vw[3]);
 }
 
-// scratch planes: ((pair_local * 2 + tensor) * 2 + (0 = U, 1 = V)) of n_half rows x 128 channels.
-__global__ void __launch_bounds__(256) fold_kernel(CacheView view, int32_t pair0, int32_t pair_count, int32_t n_in,
-                                                   int32_t n_half, int32_t sink, uint4* __restrict__ scratch)
+// One fold job: the non-sink rows of `pair_count` (batch, layer, kv_head) triples starting at
+// pair0, K and V, into the planes ((pair_local * 2 + tensor) * 2 + (0 = U, 1 = V)) of `dst`, each
+// n_half rows x 128 channels.  Item i of a job is one 16-byte vector of one folded row.
+struct FoldJob {
+    int32_t pair0, pair_count, n_in, n_half, sink;
+    uint4* dst;
+};
+
+// A job never exceeds the scratch buffer (2304 MiB, 32 bytes per item), so item counts fit 32 bits.
+__device__ __forceinline__ uint32_t fold_items(const FoldJob& job) { return (uint32_t)job.pair_count * 2u * job.n_half * 16u; }
+
+// Items i, i + stride, ... (at most B of them, below `total`): all loads first, then the stores.
+template <int B>
+__device__ __forceinline__ void fold_batch(const CacheView& view, const FoldJob& job, uint32_t i, uint32_t stride,
+                                           uint32_t total)
 {
-    const int64_t per_mat = (int64_t)n_half * 16;
-    const int64_t total = (int64_t)pair_count * 2 * per_mat;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int32_t vcol = (int32_t)(i & 15);
-        const int64_t row = i >> 4;
-        const int32_t n = (int32_t)(row % n_half);
-        const int32_t pt = (int32_t)(row / n_half);  // pair_local * 2 + tensor
-        const int32_t tensor = pt & 1;
-        const char* x = static_cast<const char*>(tensor_base(view, tensor)) +
-                        (matrix_offset(view, pair0 + (pt >> 1)) + (int64_t)sink * view.stride_token) * 2;
-        const int32_t nr = n_in - 1 - n;
-        const uint4 a = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * view.stride_token * 2) + vcol);
-        uint4 u, v;
-        if (nr != n) {
-            const uint4 b = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)nr * view.stride_token * 2) + vcol);
-            fold8(a, b, &u, &v);
-        } else {  // middle row of an odd-length signal
-            u = a;
-            v = make_uint4(0u, 0u, 0u, 0u);
+    uint4 a[B], b[B];
+    uint4* out[B];
+    bool mid[B];
+#pragma unroll
+    for (int j = 0; j < B; ++j) {
+        const uint32_t ij = i + j * stride;
+        out[j] = nullptr;
+        if (ij < total) {
+            const uint32_t vcol = ij & 15u, row = ij >> 4;
+            const uint32_t pt = row / (uint32_t)job.n_half;  // pair_local * 2 + tensor
+            const int32_t n = (int32_t)(row - pt * (uint32_t)job.n_half);
+            const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
+                            (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
+            const int32_t nr = job.n_in - 1 - n;
+            mid[j] = nr == n;  // middle row of an odd-length signal: u = x, v = 0
+            a[j] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * view.stride_token * 2) + vcol);
+            b[j] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)nr * view.stride_token * 2) + vcol);
+            out[j] = job.dst + (int64_t)row * 32 - (int64_t)n * 16 + vcol;  // plane pt * 2, row n
         }
-        uint4* pu = scratch + ((int64_t)pt * 2 * n_half + n) * 16 + vcol;
-        pu[0] = u;
-        pu[per_mat] = v;
     }
+    const int64_t plane = (int64_t)job.n_half * 16;
+#pragma unroll
+    for (int j = 0; j < B; ++j) {
+        if (out[j]) {
+            uint4 u, v;
+            fold8(a[j], b[j], &u, &v);
+            if (mid[j]) {
+                u = a[j];
+                v = make_uint4(0u, 0u, 0u, 0u);
+            }
+            out[j][0] = u;
+            out[j][plane] = v;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const FoldJob job)
+{
+    const uint32_t total = fold_items(job), stride = gridDim.x * blockDim.x;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += 4 * stride)
+        fold_batch<4>(view, job, i, stride, total);
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -484,7 +512,7 @@ bool encode_scratch_map(CUtensorMap* map, void* scratch, int32_t n_half, int32_t
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t kFoldScratchBytes = size_t(2304) << 20;  // one 7B-shaped cache of 4096 tokens fits in one pass
+constexpr size_t kFoldBufferBytes = size_t(2304) << 20;  // scratch for the folded inputs: a 7B-shaped cache of 4096 tokens fits in one pass
 
 }  // namespace
 
@@ -511,10 +539,15 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         state->attr_set = true;
     }
     const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
+    const int32_t m_tiles = (rows_half + BM - 1) / BM;
     const int32_t pairs = view.mats_per_tensor;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;  // K and V, U and V planes
-    const int32_t chunk = (int32_t)std::max<size_t>(1, std::min<size_t>(kFoldScratchBytes / per_pair, (size_t)pairs));
-    if ((size_t)chunk * per_pair > state->scratch_bytes) {
+
+    // One pass when the folded inputs fit the scratch buffer, else several passes of `chunk` pairs.
+    const int64_t fit = std::max<int64_t>(1, (int64_t)(kFoldBufferBytes / per_pair));
+    const int64_t chunk = std::min<int64_t>(fit, pairs);
+    const size_t need = (size_t)chunk * per_pair;
+    if (need > state->scratch_bytes) {
         if (state->scratch) {
             cudaError_t e = cudaDeviceSynchronize();
             if (e != cudaSuccess) return e;
@@ -522,46 +555,50 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
             state->scratch = nullptr;
             state->scratch_bytes = 0;
         }
-        const cudaError_t e = cudaMalloc(&state->scratch, (size_t)chunk * per_pair);
+        const cudaError_t e = cudaMalloc(&state->scratch, need);
         if (e != cudaSuccess) {
             state->last_error = "cudaMalloc(fold scratch)";
             return e;
         }
-        state->scratch_bytes = (size_t)chunk * per_pair;
+        state->scratch_bytes = need;
     }
     CUtensorMap map_p;
     if (!encode_basis_map(&map_p, basis)) {
         state->last_error = "tensor map encoding rejected the basis";
         return cudaErrorInvalidValue;
     }
-
-    for (int32_t p0 = 0; p0 < pairs; p0 += chunk) {
-        const int32_t count = std::min(chunk, pairs - p0);
-        CUtensorMap map_x;
-        if (!encode_scratch_map(&map_x, state->scratch, n_half, count * 4)) {
-            state->last_error = "tensor map encoding rejected the scratch planes";
-            return cudaErrorInvalidValue;
-        }
-        const int64_t items = (int64_t)count * 2 * n_half * 16;
-        const unsigned fold_grid = (unsigned)std::min<int64_t>((items + 255) / 256, (int64_t)sm_count * 16);
-        fold_kernel<<<fold_grid, 256, 0, stream>>>(view, p0, count, basis.n_in, n_half, sink,
-                                                  static_cast<uint4*>(state->scratch));
+    for (int64_t p0 = 0; p0 < pairs; p0 += chunk) {
+        FoldJob job;
+        job.pair0 = (int32_t)p0;
+        job.pair_count = (int32_t)std::min<int64_t>(chunk, pairs - p0);
+        job.n_in = basis.n_in;
+        job.n_half = n_half;
+        job.sink = sink;
+        job.dst = static_cast<uint4*>(state->scratch);
+        const int64_t items = (int64_t)job.pair_count * 2 * n_half * 16;  // < 2^31: the buffer holds at most 2304 MiB / 32 B
+        const unsigned fold_grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((items + 1023) / 1024, (int64_t)sm_count * 8));
+        fold_kernel<<<fold_grid, 256, 0, stream>>>(view, job);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) {
             state->last_error = "fold_kernel launch";
             return e;
         }
+        CUtensorMap map_x;
+        if (!encode_scratch_map(&map_x, state->scratch, n_half, job.pair_count * 4)) {
+            state->last_error = "tensor map encoding rejected the scratch planes";
+            return cudaErrorInvalidValue;
+        }
         GemmParams prm;
         prm.n_keep = basis.n_keep;
         prm.rows_half = rows_half;
         prm.basis_rows_pad = basis.fold_rows_pad;
-        prm.pair0 = p0;
-        prm.pair_count = count;
-        prm.m_tiles = (rows_half + BM - 1) / BM;
+        prm.pair0 = job.pair0;
+        prm.pair_count = job.pair_count;
+        prm.m_tiles = m_tiles;
         prm.k_steps = (n_half + BK - 1) / BK;
         prm.sink = sink;
         prm.status = status_dev;
-        const int32_t tiles = count * prm.m_tiles;
+        const int32_t tiles = job.pair_count * m_tiles;
         const int grid = std::min<int32_t>(tiles, sm_count);
         if (hooks.before) hooks.before(hooks.user, stream);
         freqkv_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_p, map_x, view, prm);

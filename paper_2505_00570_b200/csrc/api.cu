@@ -191,7 +191,7 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need
             x.ld = (n_in + 63) / 64 * 64;
             x.rows_pad = (n_keep + 63) / 64 * 64;
             x.fold_ld = ((n_in + 1) / 2 + 63) / 64 * 64;
-            x.fold_rows_pad = ((n_keep + 1) / 2 + 127) / 128 * 128;
+            x.fold_rows_pad = ((n_keep + 1) / 2 + 255) / 256 * 256;
         };
         shape(b);
         const size_t elems = (size_t)b.ld * b.rows_pad;

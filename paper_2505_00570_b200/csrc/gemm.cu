@@ -13,14 +13,21 @@
 // Two kernels per call:
 //   fold_kernel         reads every non-sink cache row once and writes U and V (bf16) to a scratch
 //                       buffer, one plane of ceil(N/2) x 128 per (matrix, u|v); HBM-bound.
-//   freqkv_gemm_kernel  one CTA per SM, persistent over output tiles of 128 folded rows x 256
-//                       columns (the K matrix and the V matrix of one (batch, layer, kv_head) side
-//                       by side, so K and V share every instruction).  Per tile it first accumulates
-//                       S = Pe U, then D = Po V, in the two halves of tensor memory:
+//   freqkv_gemm_kernel  persistent, one CTA per SM, CTAs paired into clusters of two that share
+//                       every MMA (tcgen05 cta_group::2).  A cluster works on output tiles of 256
+//                       folded rows x 256 columns (the K matrix and the V matrix of one (batch,
+//                       layer, kv_head) side by side, so K and V share every instruction): CTA r
+//                       of the pair holds rows 128 r .. 128 r + 127 of the basis slice and of the
+//                       accumulators, and HALF of the input slice (r = 0: the K channels, r = 1: the
+//                       V channels) -- the tensor cores of both SMs read both halves, so every
+//                       byte of U / V is brought into shared memory once per 256 output rows.  Per
+//                       tile the pair first accumulates S = Pe U, then D = Po V, in the two halves
+//                       of tensor memory.  In each CTA:
 //     warp 0      TMA producer: per 64-row slice of the contraction one box of Pe or Po (128 x 64)
-//                 and 4 boxes of U or V (64 rows x 64 channels), 128-byte swizzled, into a ring
-//                 of 4 stages of 48 KB;
-//     warp 1      MMA issuer: 4 tcgen05.mma (128 x 256 x 16) per stage;
+//                 and 2 boxes of U or V (64 rows x 64 channels), 128-byte swizzled, into a ring
+//                 of 6 stages of 32 KB; the bytes of both CTAs complete the leader's barrier;
+//     warp 1      MMA issuer (leader CTA only): 4 tcgen05.mma (256 x 256 x 16) per stage, commits
+//                 multicast to the barriers of both CTAs;
 //     warps 2-9   epilogue: when S is complete they park it in registers (which frees that half
 //                 of tensor memory for the next tile while D is still accumulating); when D is
 //                 complete they form s + d and s - d, round to bf16 (nearest even) and store rows
@@ -29,8 +36,9 @@
 // The kernel reads only the scratch planes and the basis, so writing the cache in place is safe.
 //
 // Every wait on an mbarrier is bounded in time: a wait that runs out sets a bit in the status
-// word, raises a CTA-wide abort flag that ends every other role's loop, the producer drains
-// its copies in flight, tensor memory is freed and the kernel returns.
+// word, raises a CTA-wide abort flag that ends every other role's loop, the producer lets its
+// copies in flight land, the two CTAs meet at a cluster barrier, tensor memory is freed and
+// the kernel returns.
 #include <cuda.h>
 
 #include <algorithm>
@@ -41,27 +49,27 @@
 namespace freqkv {
 namespace {
 
-constexpr int BM = 128;        // folded output rows per tile (one UMMA of M = 128 per accumulator); 256 columns: K | V
+constexpr int BM = 128;        // folded output rows per CTA and tile (the cluster's tile has 2 x 128); 256 columns: K | V
 constexpr int BK = 64;         // contraction slice per stage (folded rows)
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;               // 16 KB: 128 rows x 64 bf16, 128 B per row
 constexpr int B_CHUNK_BYTES = BK * 128;            // 8 KB: 64 rows x 64 channels
-constexpr int B_BYTES = 4 * B_CHUNK_BYTES;         // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 48 KB
+constexpr int B_BYTES = 2 * B_CHUNK_BYTES;         // 16 KB: this CTA's 128 of the 256 columns
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 32 KB per CTA
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int NUM_THREADS = 320;                   // 10 warps
 constexpr int EPI_WARPS = 8;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+constexpr unsigned long long LANDING_NS = 1000000ull;        // 1 ms: far longer than any copy in flight needs
 
-constexpr uint32_t ERR_FULL_WAIT = 1u, ERR_EMPTY_WAIT = 2u, ERR_ACC_FULL_WAIT = 4u, ERR_ACC_EMPTY_WAIT = 8u,
-                   ERR_DRAIN_WAIT = 16u;
+constexpr uint32_t ERR_FULL_WAIT = 1u, ERR_EMPTY_WAIT = 2u, ERR_ACC_FULL_WAIT = 4u, ERR_ACC_EMPTY_WAIT = 8u;
 
 struct GemmParams {
     int32_t n_keep;             // L
     int32_t rows_half;          // ceil(L / 2): folded output rows
     int32_t basis_rows_pad;     // row offset of the Po plane inside the basis tensor map
     int32_t pair0, pair_count;  // (batch, layer, kv_head) triples covered by this launch
-    int32_t m_tiles, k_steps;
+    int32_t m_pairs, k_steps;   // tiles of 256 folded rows per (batch, layer, kv_head); slices per phase
     int32_t sink;
     int32_t* status;
 };
@@ -85,17 +93,39 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank)
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
 }
 
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Acquire at cluster scope: some of the arrivals these waits observe come from the peer CTA.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -124,20 +154,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t c0, int32_t c1)
+// TMA loads of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on
+// the barrier `cluster_bar` of the leader CTA.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int32_t c0,
+                                            int32_t c1)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1)
         : "memory");
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t c0, int32_t c1,
-                                            int32_t c2)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int32_t c0,
+                                            int32_t c1, int32_t c2)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 
@@ -154,23 +187,30 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, A K-major, B MN-major, M = 128, N = 256.
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, A K-major, B MN-major, M = 256 (128 rows
+// in each CTA of the pair), N = 256.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((256u >> 3) << 17) |
-                           ((128u >> 4) << 24);
+                           ((256u >> 4) << 24);
 
+// Issued by one thread of the leader CTA; both CTAs' tensor cores run it, each on its 128 rows of A
+// and D, with B read from the shared memory of both.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate)
         : "memory");
 }
 
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+// When every MMA issued so far has finished, arrive on the barrier at this offset in BOTH CTAs.
+__device__ __forceinline__ void umma_commit_both(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
 }
 
 // 32 lanes x 32 consecutive columns of tensor memory into registers r[OFF .. OFF+31].
@@ -295,7 +335,8 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     uint8_t* aligned = smem_raw + (base - raw);
     uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
     const uint32_t bar0 = base + STAGES * STAGE_BYTES;
-    // barrier slots: full[0..S), empty[S..2S), then s_full, s_empty, d_full, d_empty
+    // barrier slots (same offsets in both CTAs): full[0..S) -- used in the leader only --,
+    // empty[S..2S), then s_full, s_empty, d_full, d_empty (the two *_empty used in the leader only)
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto acc_full_bar = [&](int eo) { return bar0 + 8u * (2 * STAGES + 2 * eo); };
@@ -304,38 +345,43 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int32_t total_tiles = prm.pair_count * prm.m_tiles;
+    const uint32_t rank = cluster_rank();  // 0 = leader of the pair
+    const int32_t cluster = blockIdx.x / 2, n_clusters = gridDim.x / 2;
+    const int32_t total_tiles = prm.pair_count * prm.m_pairs;  // tiles of 256 folded rows x 256 columns
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), 1);
-            mbar_init(empty_bar(s), 1);
+            mbar_init(full_bar(s), 1);   // the leader's producer arrives; both producers' bytes are counted
+            mbar_init(empty_bar(s), 1);  // one multicast commit
         }
         for (int eo = 0; eo < 2; ++eo) {
-            mbar_init(acc_full_bar(eo), 1);
-            mbar_init(acc_empty_bar(eo), EPI_WARPS);
+            mbar_init(acc_full_bar(eo), 1);               // one multicast commit
+            mbar_init(acc_empty_bar(eo), 2 * EPI_WARPS);  // the epilogue warps of both CTAs
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {  // tensor memory: all 512 columns (S in 0..255, D in 256..511)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    if (warp == 1) {  // tensor memory of the pair: all 512 columns in each CTA (S in 0..255, D in 256..511)
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
             uint32_t it = 0;  // global slice counter: stage = it % STAGES, phase = it / STAGES
             bool alive = true;
-            for (int32_t tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x) {
-                const int32_t pair_local = tile / prm.m_tiles, mt = tile % prm.m_tiles;
+            for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters) {
+                const int32_t pair_local = tile / prm.m_pairs;
+                const int32_t m0 = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM;
                 for (int eo = 0; eo < 2 && alive; ++eo) {
+                    const int32_t plane = (pair_local * 2 + (int32_t)rank) * 2 + eo;  // rank 0: K channels, rank 1: V
                     for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
                         const int s = it % STAGES;
                         if (it >= STAGES &&
@@ -344,35 +390,28 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                             break;
                         }
                         const uint32_t stage = base + s * STAGE_BYTES;
-                        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+                        const uint32_t leader_full = cluster_addr(full_bar(s), 0);
+                        if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
                         const int32_t k0 = ks * BK;
-                        tma_load_2d(stage, &map_p, full_bar(s), k0, eo * prm.basis_rows_pad + mt * BM);
-                        const uint32_t bs = stage + A_BYTES;
-                        const int32_t plane_k = (pair_local * 2 + 0) * 2 + eo, plane_v = (pair_local * 2 + 1) * 2 + eo;
-                        tma_load_3d(bs + 0 * B_CHUNK_BYTES, &map_x, full_bar(s), 0, k0, plane_k);
-                        tma_load_3d(bs + 1 * B_CHUNK_BYTES, &map_x, full_bar(s), 64, k0, plane_k);
-                        tma_load_3d(bs + 2 * B_CHUNK_BYTES, &map_x, full_bar(s), 0, k0, plane_v);
-                        tma_load_3d(bs + 3 * B_CHUNK_BYTES, &map_x, full_bar(s), 64, k0, plane_v);
+                        tma_load_2d(stage, &map_p, leader_full, k0, eo * prm.basis_rows_pad + m0);
+                        tma_load_3d(stage + A_BYTES, &map_x, leader_full, 0, k0, plane);
+                        tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, &map_x, leader_full, 64, k0, plane);
                     }
                 }
             }
-            if (*abort_flag) {
-                // drain: every slice issued but possibly not yet landed completes its full barrier
-                const uint32_t first = it > STAGES ? it - STAGES : 0;
-                for (uint32_t j = first; j < it; ++j) {
-                    int dummy = 0;
-                    mbar_wait(full_bar(j % STAGES), (j / STAGES) & 1, &dummy, prm.status, ERR_DRAIN_WAIT);
-                }
+            if (*abort_flag) {  // let the copies in flight land before this CTA's shared memory goes away
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < LANDING_NS) __nanosleep(1000);
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0, tile_no = 0;
             bool alive = true;
-            for (int32_t tile = blockIdx.x; tile < total_tiles && alive; tile += gridDim.x, ++tile_no) {
+            for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters, ++tile_no) {
                 for (int eo = 0; eo < 2 && alive; ++eo) {
-                    if (tile_no > 0) {  // this accumulator must have been read by the epilogue of the last tile
+                    if (tile_no > 0) {  // both CTAs' epilogues must have read this accumulator of the last tile
                         if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT)) {
                             alive = false;
                             break;
@@ -389,24 +428,25 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         const uint32_t a0 = base + s * STAGE_BYTES, b0 = a0 + A_BYTES;
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; ++kk) {
-                            // A: 128 rows, 8-row groups 1 KB apart; 16 k-elements = 32 bytes inside the swizzled row
+                            // A: 128 rows per CTA, 8-row groups 1 KB apart; 16 k-elements = 32 bytes inside the swizzled row
                             const uint64_t ad = smem_desc(a0 + kk * 32, 16, 1024);
-                            // B: 4 chunks of 64 channels 8 KB apart (leading offset), 8-row groups 1 KB apart
+                            // B: per CTA 2 chunks of 64 channels 8 KB apart (leading offset), 8-row groups 1 KB apart
                             const uint64_t bd = smem_desc(b0 + kk * 2048, B_CHUNK_BYTES, 1024);
                             umma_bf16(tmem_base + eo * 256, ad, bd, (ks | kk) != 0);
                         }
-                        umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+                        umma_commit_both(empty_bar(s));  // frees the stage in both CTAs when these MMAs have read it
                     }
-                    if (alive) umma_commit(acc_full_bar(eo));
+                    if (alive) umma_commit_both(acc_full_bar(eo));
                 }
             }
         }
     } else {
-        // ---------------- epilogue ----------------
+        // ---------------- epilogue (both CTAs, each on its own 128 rows) ----------------
         const int ew = warp - 2, quarter = warp % 4, tensor = ew / 4;  // tensor: 0 = K columns, 1 = V columns
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tensor * 128;
+        const uint32_t leader_s_empty = cluster_addr(acc_empty_bar(0), 0), leader_d_empty = cluster_addr(acc_empty_bar(1), 0);
         uint32_t tile_no = 0;
-        for (int32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_no) {
+        for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
             // S = Pe U: park this thread's row (128 columns) in registers, release that half
             if (!mbar_wait(acc_full_bar(0), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -418,13 +458,13 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(0));
+            if (lane == 0) mbar_arrive_cluster(leader_s_empty);
 
             // D = Po V: combine and store rows m and L-1-m
             if (!mbar_wait(acc_full_bar(1), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int32_t pair_local = tile / prm.m_tiles, mt = tile % prm.m_tiles;
-            const int32_t m = mt * BM + quarter * 32 + lane;
+            const int32_t pair_local = tile / prm.m_pairs;
+            const int32_t m = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
             const int32_t mr = prm.n_keep - 1 - m;
             const bool row_ok = m < prm.rows_half;
             __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
@@ -455,15 +495,17 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(1));
+            if (lane == 0) mbar_arrive_cluster(leader_d_empty);
         }
     }
 
+    // Neither CTA may leave (its barriers and tensor memory are used by the other) before both are done.
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    cluster_sync_all();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
     }
 }
 
@@ -536,10 +578,29 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
             state->last_error = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
         }
+        // how many CTA pairs the device can hold at once (one CTA per SM; SMs pair up inside a GPC)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * (sm_count / 2)));
+        cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        const cudaError_t q = cudaOccupancyMaxActiveClusters(&n, freqkv_gemm_kernel, &cfg);
+        if (q != cudaSuccess || n < 1) {
+            state->last_error = "cudaOccupancyMaxActiveClusters: no CTA pair fits on this device";
+            return q != cudaSuccess ? q : cudaErrorLaunchOutOfResources;
+        }
+        state->max_clusters = std::min(n, sm_count / 2);
         state->attr_set = true;
     }
     const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
-    const int32_t m_tiles = (rows_half + BM - 1) / BM;
+    const int32_t m_pairs = (rows_half + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
     const int32_t pairs = view.mats_per_tensor;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;  // K and V, U and V planes
 
@@ -594,15 +655,26 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         prm.basis_rows_pad = basis.fold_rows_pad;
         prm.pair0 = job.pair0;
         prm.pair_count = job.pair_count;
-        prm.m_tiles = m_tiles;
+        prm.m_pairs = m_pairs;
         prm.k_steps = (n_half + BK - 1) / BK;
         prm.sink = sink;
         prm.status = status_dev;
-        const int32_t tiles = job.pair_count * m_tiles;
-        const int grid = std::min<int32_t>(tiles, sm_count);
+        const int32_t tiles = job.pair_count * m_pairs;
+        const int clusters = std::min<int32_t>(tiles, state->max_clusters);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * clusters));
+        cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
         if (hooks.before) hooks.before(hooks.user, stream);
-        freqkv_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_p, map_x, view, prm);
-        e = cudaGetLastError();
+        e = cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel, map_p, map_x, view, prm);
         if (hooks.after) hooks.after(hooks.user, stream);
         if (e != cudaSuccess) {
             state->last_error = "freqkv_gemm_kernel launch";

@@ -8,6 +8,7 @@ struct GemmState {
     const char* last_error = nullptr;
     int kernels_last_call = 0;
     bool attr_set = false;
+    int max_clusters = 0;     // CTA pairs that can be resident at once
     void* scratch = nullptr;  // folded inputs U, V: [pairs][K|V][U|V][ceil(n_in/2)][128] bf16 per pass
     size_t scratch_bytes = 0;
 };

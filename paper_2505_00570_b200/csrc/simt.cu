@@ -4,6 +4,8 @@
 // output with a classic shared-memory tiled product; results go to a scratch buffer and a
 // second kernel copies them over rows [sink, sink + L) of the cache, because every output row
 // depends on every input row of the same matrix and the two ranges overlap.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace freqkv {
@@ -145,6 +147,42 @@ __global__ void append_kernel(CacheView view, int32_t batch, AppendLens lens, in
     }
 }
 
+// Many new rows per matrix (prefill chunks): one block column per matrix, so that the matrix
+// arithmetic is done once per thread and each thread then moves four 16-byte vectors per round,
+// loads first.  Block (x, y): matrix x (K matrices first, then V), y-th share of its vectors.
+__global__ void __launch_bounds__(256) append_rows_kernel(CacheView view, int32_t batch, AppendLens lens, int32_t n_new,
+                                                          int32_t elt_size, const uint4* __restrict__ new_k,
+                                                          const uint4* __restrict__ new_v)
+{
+    const uint32_t vec_per_row = (uint32_t)(view.head_dim * elt_size / 16);
+    const uint32_t row_stride = (uint32_t)(view.stride_token * elt_size / 16);  // vectors between cache rows
+    const int32_t mats = batch * view.layers * view.kv_heads;
+    const int32_t tensor = (int32_t)blockIdx.x >= mats;
+    const int32_t idx = (int32_t)blockIdx.x - tensor * mats;
+    const int32_t b = idx / (view.layers * view.kv_heads);
+    const uint32_t total = (uint32_t)n_new * vec_per_row;
+    const uint4* src = (tensor ? new_v : new_k) + (int64_t)idx * total;
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(tensor_base(view, tensor)) +
+                                          (matrix_offset(view, idx) + (int64_t)lens.len[b] * view.stride_token) * elt_size);
+    const uint32_t stride = gridDim.y * blockDim.x;
+    for (uint32_t i0 = blockIdx.y * blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = i0 + j * stride;
+            if (i < total) v[j] = __ldg(src + i);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = i0 + j * stride;
+            if (i < total) {
+                const uint32_t r = i / vec_per_row, vcol = i - r * vec_per_row;
+                dst[(size_t)r * row_stride + vcol] = v[j];
+            }
+        }
+    }
+}
+
 unsigned grid_for(int64_t work_items, int threads)
 {
     int64_t blocks = (work_items + threads - 1) / threads;
@@ -196,7 +234,14 @@ cudaError_t launch_append(const CacheView& view, int32_t dtype, int32_t batch, c
         sub.batch0 = view.batch0 + b0;
         const uint4* nk = static_cast<const uint4*>(new_k) + (int64_t)b0 * seq_vecs;
         const uint4* nv = static_cast<const uint4*>(new_v) + (int64_t)b0 * seq_vecs;
-        append_kernel<<<grid_for(2 * nb * seq_vecs, 256), 256, 0, stream>>>(sub, nb, lens, n_new, elt, nk, nv);
+        const int64_t mat_vecs = (int64_t)n_new * row_vecs;  // per matrix
+        const int64_t mats2 = (int64_t)2 * nb * view.layers * view.kv_heads;
+        if (mat_vecs >= 4096 && mat_vecs < ((int64_t)1 << 31) && mats2 < ((int64_t)1 << 31)) {
+            const unsigned gy = (unsigned)std::min<int64_t>((mat_vecs + 1023) / 1024, 64);
+            append_rows_kernel<<<dim3((unsigned)mats2, gy), 256, 0, stream>>>(sub, nb, lens, n_new, elt, nk, nv);
+        } else {
+            append_kernel<<<grid_for(2 * nb * seq_vecs, 256), 256, 0, stream>>>(sub, nb, lens, n_new, elt, nk, nv);
+        }
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }

@@ -101,6 +101,34 @@ def test_append_rows_and_capacity(ctx):
     assert torch.equal(k[2, :, :, 35:40], nk[2])  # a refused append wrote nothing
 
 
+@pytest.mark.parametrize("dtype,row_pad", [(torch.bfloat16, 0), (torch.bfloat16, 8), (torch.float32, 0)])
+def test_append_large_chunk(ctx, dtype, row_pad):
+    """A prefill-sized chunk (hundreds of rows per matrix) takes the per-matrix copy kernel:
+    rows land at each sequence's own length, every other byte (padding and canaries included)
+    keeps its value."""
+    w = small(cap=700, dtype=dtype, B=2, Ly=2, H=3, sink=4)
+    (kbuf, k), (vbuf, v) = parity.guarded_cache(w, torch.device("cuda"), fill_len=700, row_pad=row_pad)
+    kbuf0, vbuf0 = kbuf.clone(), vbuf.clone()
+    n_new = 333
+    nk = torch.randn(2, 2, 3, n_new, 128, device="cuda").to(dtype)
+    nv = torch.randn(2, 2, 3, n_new, 128, device="cuda").to(dtype)
+    starts = [0, 367]
+    lens = ctx.append(k, v, nk, nv, starts)
+    assert lens == [n_new, 700]
+    for b, start in enumerate(starts):
+        assert torch.equal(k[b, :, :, start:start + n_new], nk[b]) and torch.equal(v[b, :, :, start:start + n_new], nv[b])
+    # restore the appended rows: the buffers must then equal their pre-call copies bit for bit
+    k0 = kbuf0[parity.GUARD:parity.GUARD + k.shape[0] * k.shape[1] * k.shape[2] * 700 * (128 + row_pad)].view(2, 2, 3, 700, 128 + row_pad)[..., :128]
+    v0 = vbuf0[parity.GUARD:parity.GUARD + k.shape[0] * k.shape[1] * k.shape[2] * 700 * (128 + row_pad)].view(2, 2, 3, 700, 128 + row_pad)[..., :128]
+    for b, start in enumerate(starts):
+        k[b, :, :, start:start + n_new] = k0[b, :, :, start:start + n_new]
+        v[b, :, :, start:start + n_new] = v0[b, :, :, start:start + n_new]
+    assert torch.equal(kbuf.view(torch.int16 if dtype == torch.bfloat16 else torch.int32),
+                       kbuf0.view(torch.int16 if dtype == torch.bfloat16 else torch.int32))
+    assert torch.equal(vbuf.view(torch.int16 if dtype == torch.bfloat16 else torch.int32),
+                       vbuf0.view(torch.int16 if dtype == torch.bfloat16 else torch.int32))
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_iterative_stream_matches_oracle(ctx, dtype):
     """Tokens enter one at a time; a full cache is compressed to half its non-sink length

@@ -167,10 +167,14 @@ def stream(tokens, capacity: int, sink: int, retain: float = 0.5) -> tuple[np.nd
     d = tokens.shape[1]
     cache = np.zeros((capacity, d), dtype=np.float64)
     length, count = 0, 0
+    L = int(np.floor(retain * (capacity - sink)))
     for row in tokens:
         if length == capacity:
-            L = int(np.floor(retain * (capacity - sink)))
-            cache, length = compress_cache(cache, length, L, sink)
+            # same steps as compress_cache / append above, written on the one array in place
+            # (a stream of 10^5 tokens would otherwise copy the whole cache once per token)
+            cache[sink:sink + L, :] = compress_matrix(cache[sink:length, :], L)
+            length = sink + L
             count += 1
-        cache, length = append(cache, row[None, :], length)
+        cache[length, :] = row
+        length += 1
     return cache, length, count

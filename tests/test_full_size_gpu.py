@@ -1,0 +1,207 @@
+"""GPU parity at the full sizes of the five benchmark configurations, in the launch
+configuration ``bench.py`` times (variant AUTO, whole caches in one call).
+
+The oracle cannot recompute a whole multi-gigabyte cache in reasonable time, so each test
+compares a seeded sample of matrices with it -- always the first and the last matrix, for the
+ragged batch the shortest and the longest sequence too -- on bit-identical inputs copied back
+from the device, and checks the properties that hold for every matrix on the device itself:
+sink rows and rows past the new length keep their bytes, lengths and compression counts are
+the ones the trigger rule gives.  Tolerance: relative L2 <= 1e-2 per matrix (bf16 caches); for
+streams, where the oracle compresses its own unrounded state, times sqrt(number of compressions).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_00570_b200 import binding as fk
+from paper_2505_00570_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 1e-2
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = fk.Context(0)
+    c.set_variant(fk.AUTO)
+    yield c
+    c.close()
+
+
+def need_gib(gib: float):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gib * 2**30:
+        pytest.skip(f"needs {gib:.0f} GiB of free device memory")
+
+
+def coords(i: int, shape) -> tuple[int, int, int, int]:
+    """Matrix index (K matrices first, then V) -> (tensor, batch, layer, kv_head)."""
+    B, Ly, H = shape[0], shape[1], shape[2]
+    per = B * Ly * H
+    t, j = divmod(i, per)
+    return t, j // (Ly * H), (j // H) % Ly, j % H
+
+
+def check_uniform(ctx, name: str, sample: int):
+    w = synth.WORKLOADS[name]
+    cache_len, sink = w.capacity, w.sink
+    kept = w.kept_len(cache_len)
+    k, v = synth.make_cache(w, "cuda")
+    ids = synth.sample_matrix_ids(w.n_matrices, sample, w.seed + 5)
+    inputs = {}
+    for i in ids:
+        t, b, l, h = coords(i, k.shape)
+        inputs[i] = parity.to_f64((k, v)[t][b, l, h, sink:cache_len])
+    # device-side copies of what must not change: sink rows and the rows past the new length
+    head = [t[..., :sink, :].clone() for t in (k, v)]
+    tail = [t[..., sink + kept:, :].clone() for t in (k, v)]
+    assert ctx.resolve_variant(fk.layout_of(k), cache_len - sink, kept) == fk.GEMM
+    new_len = ctx.compress(k, v, cache_len, kept, sink)
+    assert ctx.last_device_status() == fk.OK and new_len == sink + kept
+    for t, hd, tl in zip((k, v), head, tail):
+        assert torch.equal(t[..., :sink, :], hd), "sink rows changed"
+        assert torch.equal(t[..., sink + kept:, :], tl), "rows past the new length changed"
+    worst = 0.0
+    for i in ids:
+        t, b, l, h = coords(i, k.shape)
+        want = oracle.compress_matrix(inputs[i], kept)
+        got = parity.to_f64((k, v)[t][b, l, h, sink:sink + kept])
+        worst = max(worst, parity.rel_l2(got, want))
+    assert worst <= TOL_BF16, f"{name}: relative L2 {worst:.3e}"
+    return worst
+
+
+def test_config2_llama2_7b_full(ctx):
+    """32 x 32 heads x 128, 4096 tokens, 4 sinks, 4092 -> 2046: 2048 matrices in one call."""
+    need_gib(20)
+    check_uniform(ctx, "llama2_7b", sample=24)
+
+
+def test_config3_llama3_8b_full(ctx):
+    """Batch 8, 32 x 8 KV heads x 128, 8192 tokens, 8188 -> 4094: 4096 matrices in one call."""
+    need_gib(40)
+    check_uniform(ctx, "llama3_8b", sample=10)
+
+
+def test_config5b_ragged_full(ctx):
+    """Batch 32 of caches with seeded lengths in [1024, 8192], each compressed to half its own
+    non-sink length by one freqkv_compress_ragged call."""
+    need_gib(90)
+    w = synth.WORKLOADS["ragged_8b"]
+    sink = w.sink
+    lens = synth.ragged_lengths(w)
+    kept = [(n - sink) // 2 for n in lens]
+    k, v = synth.make_cache(w, "cuda")
+    k_in, v_in = k.clone(), v.clone()
+    new_lens = ctx.compress_ragged(k, v, lens, kept, sink)
+    assert ctx.last_device_status() == fk.OK
+    assert new_lens == [sink + x for x in kept]
+    for b in range(w.batch):
+        for t_in, t_out in ((k_in, k), (v_in, v)):
+            assert torch.equal(t_out[b, :, :, :sink], t_in[b, :, :, :sink])
+            assert torch.equal(t_out[b, :, :, sink + kept[b]:], t_in[b, :, :, sink + kept[b]:])
+    gen = torch.Generator().manual_seed(w.seed + 9)
+    seqs = {min(range(w.batch), key=lambda b: lens[b]), max(range(w.batch), key=lambda b: lens[b]), 0, w.batch - 1}
+    seqs |= set(torch.randperm(w.batch, generator=gen)[:3].tolist())
+    worst = 0.0
+    for b in sorted(seqs):
+        for (l, h) in ((0, 0), (w.layers - 1, w.kv_heads - 1)):
+            for t_in, t_out in ((k_in, k), (v_in, v)):
+                want = oracle.compress_matrix(parity.to_f64(t_in[b, l, h, sink:lens[b]]), kept[b])
+                got = parity.to_f64(t_out[b, l, h, sink:sink + kept[b]])
+                worst = max(worst, parity.rel_l2(got, want))
+    assert worst <= TOL_BF16, f"ragged: relative L2 {worst:.3e}"
+
+
+def test_config4_decode_stream_full(ctx):
+    """Batch 16 of 7B-shaped caches, 32768 tokens appended one per step from empty caches; a
+    full cache is compressed (4092 -> 2046) before the next token goes in: 15 compressions."""
+    need_gib(60)
+    w = synth.WORKLOADS["stream_7b"]
+    cap, sink, total = w.capacity, w.sink, 32768
+    kept = w.kept_len(cap)
+    k, v = synth.make_cache(w, "cuda", fill_len=0)
+    ids = synth.sample_matrix_ids(w.n_matrices, 4, w.seed + 5)
+    where = [coords(i, k.shape) for i in ids]
+    gens, scales, state = [], [], [None, None]
+    for which in range(2):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed + 1000 * which)
+        gens.append(g)
+        scales.append(synth.channel_scales(w, g, "cuda"))
+    record = [np.empty((total, w.head_dim)) for _ in ids]
+    lens, count = [0] * w.batch, 0
+    block = 64
+    for t0 in range(0, total, block):
+        rows = []
+        for which in range(2):
+            r, state[which] = synth.ar1_rows(w, block, gens[which], "cuda", scales[which], state[which])
+            rows.append(r)
+        for n, (t, b, l, h) in enumerate(where):
+            record[n][t0:t0 + block] = parity.to_f64(rows[t][b, l, h])
+        for j in range(block):
+            nk, nv = rows[0][:, :, :, j:j + 1].contiguous(), rows[1][:, :, :, j:j + 1].contiguous()
+            try:
+                lens = ctx.append(k, v, nk, nv, lens)
+            except fk.FreqKVError as e:
+                assert e.status == fk.ERR_CAPACITY
+                new_len = ctx.compress(k, v, cap, kept, sink)
+                count += 1
+                lens = ctx.append(k, v, nk, nv, [new_len] * w.batch)
+    assert ctx.last_device_status() == fk.OK
+    assert count == 15 == oracle.compression_count(total, cap, sink, kept)  # the paper's count for 32K tokens
+    tol = TOL_BF16 * count ** 0.5
+    for n, (t, b, l, h) in enumerate(where):
+        want, length, c = oracle.stream(record[n], cap, sink, 0.5)
+        assert length == lens[b] and c == count
+        got = parity.to_f64((k, v)[t][b, l, h, :length])
+        assert np.array_equal(got[:sink], want[:sink])
+        assert parity.rel_l2(got, want[:length]) < tol
+
+
+def test_config5a_chunked_prefill_full(ctx):
+    """One 7B-shaped sequence of 262144 tokens fed in 4096-token chunks; every fill triggers a
+    compression 4092 -> 2046: 127 of them, the paper's count for 256K tokens."""
+    need_gib(30)
+    w = synth.WORKLOADS["prefill_7b"]
+    cap, sink, total, chunk = w.capacity, w.sink, 262144, 4096
+    kept = w.kept_len(cap)
+    k, v = synth.make_cache(w, "cuda", fill_len=0)
+    ids = [0, w.n_matrices - 1]
+    where = [coords(i, k.shape) for i in ids]
+    gens, scales, state = [], [], [None, None]
+    for which in range(2):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed + 1000 * which)
+        gens.append(g)
+        scales.append(synth.channel_scales(w, g, "cuda"))
+    record = [np.empty((total, w.head_dim)) for _ in ids]
+    length, count = 0, 0
+    for t0 in range(0, total, chunk):
+        rows = []
+        for which in range(2):
+            r, state[which] = synth.ar1_rows(w, chunk, gens[which], "cuda", scales[which], state[which])
+            rows.append(r)
+        for n, (t, b, l, h) in enumerate(where):
+            record[n][t0:t0 + chunk] = parity.to_f64(rows[t][b, l, h])
+        off = 0
+        while off < chunk:
+            if length == cap:
+                length = ctx.compress(k, v, cap, kept, sink)
+                count += 1
+            n_new = min(chunk - off, cap - length)
+            nk, nv = rows[0][:, :, :, off:off + n_new].contiguous(), rows[1][:, :, :, off:off + n_new].contiguous()
+            length = ctx.append(k, v, nk, nv, [length])[0]
+            off += n_new
+    assert ctx.last_device_status() == fk.OK
+    assert count == 127 == oracle.compression_count(total, cap, sink, kept)
+    tol = TOL_BF16 * count ** 0.5
+    for n, (t, b, l, h) in enumerate(where):
+        want, n_len, c = oracle.stream(record[n], cap, sink, 0.5)
+        assert n_len == length and c == count
+        got = parity.to_f64((k, v)[t][b, l, h, :length])
+        assert np.array_equal(got[:sink], want[:sink])
+        assert parity.rel_l2(got, want[:length]) < tol

@@ -268,61 +268,50 @@ __device__ __forceinline__ void fold8(const uint4& a, const uint4& b, uint4* u, 
 
 // One fold job: the non-sink rows of `pair_count` (batch, layer, kv_head) triples starting at
 // pair0, K and V, into the planes ((pair_local * 2 + tensor) * 2 + (0 = U, 1 = V)) of `dst`, each
-// n_half rows x 128 channels.  Item i of a job is one 16-byte vector of one folded row.
+// n_half rows x 128 channels (16 vectors of 16 bytes per row).
 struct FoldJob {
     int32_t pair0, pair_count, n_in, n_half, sink;
     uint4* dst;
 };
 
-// A job never exceeds the scratch buffer (2304 MiB, 32 bytes per item), so item counts fit 32 bits.
-__device__ __forceinline__ uint32_t fold_items(const FoldJob& job) { return (uint32_t)job.pair_count * 2u * job.n_half * 16u; }
-
-// Items i, i + stride, ... (at most B of them, below `total`): all loads first, then the stores.
-template <int B>
-__device__ __forceinline__ void fold_batch(const CacheView& view, const FoldJob& job, uint32_t i, uint32_t stride,
-                                           uint32_t total)
-{
-    uint4 a[B], b[B];
-    uint4* out[B];
-    bool mid[B];
-#pragma unroll
-    for (int j = 0; j < B; ++j) {
-        const uint32_t ij = i + j * stride;
-        out[j] = nullptr;
-        if (ij < total) {
-            const uint32_t vcol = ij & 15u, row = ij >> 4;
-            const uint32_t pt = row / (uint32_t)job.n_half;  // pair_local * 2 + tensor
-            const int32_t n = (int32_t)(row - pt * (uint32_t)job.n_half);
-            const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
-                            (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
-            const int32_t nr = job.n_in - 1 - n;
-            mid[j] = nr == n;  // middle row of an odd-length signal: u = x, v = 0
-            a[j] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * view.stride_token * 2) + vcol);
-            b[j] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)nr * view.stride_token * 2) + vcol);
-            out[j] = job.dst + (int64_t)row * 32 - (int64_t)n * 16 + vcol;  // plane pt * 2, row n
-        }
-    }
-    const int64_t plane = (int64_t)job.n_half * 16;
-#pragma unroll
-    for (int j = 0; j < B; ++j) {
-        if (out[j]) {
-            uint4 u, v;
-            fold8(a[j], b[j], &u, &v);
-            if (mid[j]) {
-                u = a[j];
-                v = make_uint4(0u, 0u, 0u, 0u);
-            }
-            out[j][0] = u;
-            out[j][plane] = v;
-        }
-    }
-}
-
+// Block (x, y): matrix x of the job (pair_local * 2 + tensor), y-th share of its n_half * 16 vectors.
+// The matrix arithmetic is done once per thread; each thread then folds four vectors per round,
+// all eight loads first.  Reads and writes are streaming (each byte is touched once).
 __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const FoldJob job)
 {
-    const uint32_t total = fold_items(job), stride = gridDim.x * blockDim.x;
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += 4 * stride)
-        fold_batch<4>(view, job, i, stride, total);
+    const uint32_t pt = blockIdx.x;
+    const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
+                    (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
+    const int64_t row_bytes = view.stride_token * 2;
+    const uint32_t total = (uint32_t)job.n_half * 16u, stride = gridDim.y * blockDim.x;
+    uint4* u_plane = job.dst + (int64_t)pt * 2 * total;
+    for (uint32_t i0 = blockIdx.y * blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = i0 + j * stride;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4), nr = job.n_in - 1 - n;
+                a[j] = __ldcs(reinterpret_cast<const uint4*>(x + n * row_bytes) + (i & 15u));
+                b[j] = __ldcs(reinterpret_cast<const uint4*>(x + nr * row_bytes) + (i & 15u));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = i0 + j * stride;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4);
+                uint4 u, v;
+                fold8(a[j], b[j], &u, &v);
+                if (job.n_in - 1 - n == n) {  // middle row of an odd-length signal: u = x, v = 0
+                    u = a[j];
+                    v = make_uint4(0u, 0u, 0u, 0u);
+                }
+                __stcs(u_plane + i, u);
+                __stcs(u_plane + total + i, v);
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -636,9 +625,8 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         job.n_half = n_half;
         job.sink = sink;
         job.dst = static_cast<uint4*>(state->scratch);
-        const int64_t items = (int64_t)job.pair_count * 2 * n_half * 16;  // < 2^31: the buffer holds at most 2304 MiB / 32 B
-        const unsigned fold_grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((items + 1023) / 1024, (int64_t)sm_count * 8));
-        fold_kernel<<<fold_grid, 256, 0, stream>>>(view, job);
+        const unsigned fold_y = (unsigned)std::min<int64_t>(((int64_t)n_half * 16 + 1023) / 1024, 64);
+        fold_kernel<<<dim3((unsigned)job.pair_count * 2, fold_y), 256, 0, stream>>>(view, job);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) {
             state->last_error = "fold_kernel launch";

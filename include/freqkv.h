@@ -128,9 +128,11 @@ freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* 
  * host memory.  Rows [sink, cache_len) of every matrix are copied to a device staging cache the
  * context owns (allocated on first use, same layout), compressed there exactly as
  * freqkv_compress does, and rows [sink, sink+kept_len) are copied back over the host rows.
- * All copies and kernels are enqueued on `cuda_stream`; the host buffers must stay valid and
- * untouched until that stream has been synchronised.  h2d_bytes / d2h_bytes (optional, may be
- * NULL) receive the bytes moved each way. */
+ * The work is pipelined over groups of layers on three streams the context owns (copy in,
+ * compress, copy out overlap; both directions of the bus are used at once); it starts after
+ * everything enqueued on `cuda_stream` so far, and work enqueued on `cuda_stream` afterwards starts
+ * after it.  The host buffers must stay valid and untouched until that stream has been
+ * synchronised.  h2d_bytes / d2h_bytes (optional, may be NULL) receive the bytes moved each way. */
 freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout, void* k_host, void* v_host,
                                    int32_t cache_len, int32_t kept_len, int32_t sink, void* cuda_stream,
                                    int64_t* h2d_bytes, int64_t* d2h_bytes);

@@ -36,6 +36,9 @@ struct freqkv_ctx {
     // host-buffer entry point: device staging caches
     void* stage[2] = {nullptr, nullptr};
     size_t stage_bytes = 0;
+    cudaStream_t pipe[3] = {nullptr, nullptr, nullptr};  // copy in, compress, copy out
+    cudaEvent_t pipe_begin = nullptr, pipe_end = nullptr;
+    std::vector<cudaEvent_t> pipe_events;                // per group: copied in, compressed
 };
 
 namespace {
@@ -426,6 +429,11 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     for (int i = 0; i < 2; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    for (int i = 0; i < 3; ++i)
+        if (ctx->pipe[i]) cudaStreamDestroy(ctx->pipe[i]);
+    if (ctx->pipe_begin) cudaEventDestroy(ctx->pipe_begin);
+    if (ctx->pipe_end) cudaEventDestroy(ctx->pipe_end);
+    for (auto ev : ctx->pipe_events) cudaEventDestroy(ev);
     for (auto* list : {&ctx->pending, &ctx->spare})
         for (auto& ev : *list) {
             cudaEventDestroy(ev.first);
@@ -607,43 +615,76 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
         FREQKV_CUDA(ctx, cudaMalloc(&ctx->stage[1], bytes));
         ctx->stage_bytes = bytes;
     }
-    // One 2-D copy per (tensor, batch, layer): `kv_heads` runs of rows, one run per head.  Rows of
-    // a matrix are contiguous when stride_token == head_dim; padded rows are copied with their
-    // padding (same layout on both sides).
+    // head stride below one matrix's rows (heads interleaved inside the token axis) is not
+    // something a 2-D copy can express
     const size_t row_bytes = (size_t)l.stride_token * elt;
-    auto copy_rows = [&](bool to_device, int32_t row0, int32_t rows, int64_t* counter) -> cudaError_t {
+    if (l.kv_heads > 1 && (size_t)l.stride_head * elt < (size_t)(n_in - 1) * row_bytes + (size_t)l.head_dim * elt)
+        return FREQKV_ERR_UNSUPPORTED;
+
+    // Three-deep pipeline over groups of layers: the host->device copy of group g+1, the
+    // compression of group g and the device->host copy of group g-1 run at the same time on three
+    // streams of the context (PCIe carries both directions at once), ordered by events; the
+    // caller's stream is the entry and the exit of the whole pipeline.
+    if (!ctx->pipe[0]) {
+        for (int i = 0; i < 3; ++i) FREQKV_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->pipe[i], cudaStreamNonBlocking));
+        FREQKV_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pipe_begin, cudaEventDisableTiming));
+        FREQKV_CUDA(ctx, cudaEventCreateWithFlags(&ctx->pipe_end, cudaEventDisableTiming));
+    }
+    const int32_t per_group = std::max(1, (l.layers + 7) / 8);  // layers per group: about 8 groups per sequence
+    const int32_t groups_per_seq = (l.layers + per_group - 1) / per_group;
+    const size_t n_groups = (size_t)l.batch * groups_per_seq;
+    while (ctx->pipe_events.size() < 2 * n_groups) {
+        cudaEvent_t ev;
+        FREQKV_CUDA(ctx, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        ctx->pipe_events.push_back(ev);
+    }
+    // One 2-D copy per (tensor, layer): `kv_heads` runs of rows, one run per head.  Rows of a
+    // matrix are contiguous when stride_token == head_dim; padded rows are copied with their
+    // padding (same layout on both sides).
+    auto copy_rows = [&](bool to_device, int32_t b, int32_t y0, int32_t ny, int32_t row0, int32_t rows, cudaStream_t s,
+                         int64_t* counter) -> cudaError_t {
         const size_t width = rows == 0 ? 0 : (size_t)(rows - 1) * row_bytes + (size_t)l.head_dim * elt;
+        const size_t pitch = l.kv_heads == 1 ? width : (size_t)l.stride_head * elt;
         for (int t = 0; t < 2; ++t) {
             char* host = static_cast<char*>(t ? v_host : k_host);
             char* dev = static_cast<char*>(ctx->stage[t]);
-            for (int32_t b = 0; b < l.batch; ++b)
-                for (int32_t y = 0; y < l.layers; ++y) {
-                    const size_t off = ((size_t)b * l.stride_batch + (size_t)y * l.stride_layer + (size_t)row0 * l.stride_token) * elt;
-                    const size_t pitch = (size_t)l.stride_head * elt;
-                    cudaError_t e;
-                    if (l.kv_heads == 1 || pitch >= width)
-                        e = cudaMemcpy2DAsync(to_device ? dev + off : host + off, l.kv_heads == 1 ? width : pitch,
-                                              to_device ? host + off : dev + off, l.kv_heads == 1 ? width : pitch, width,
-                                              l.kv_heads, to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost,
-                                              stream);
-                    else
-                        e = cudaErrorInvalidValue;
-                    if (e != cudaSuccess) return e;
-                    if (counter) *counter += (int64_t)width * l.kv_heads;
-                }
+            for (int32_t y = y0; y < y0 + ny; ++y) {
+                const size_t off = ((size_t)b * l.stride_batch + (size_t)y * l.stride_layer + (size_t)row0 * l.stride_token) * elt;
+                const cudaError_t e = cudaMemcpy2DAsync(to_device ? dev + off : host + off, pitch,
+                                                        to_device ? host + off : dev + off, pitch, width, l.kv_heads,
+                                                        to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost, s);
+                if (e != cudaSuccess) return e;
+                if (counter) *counter += (int64_t)width * l.kv_heads;
+            }
         }
         return cudaSuccess;
     };
-    // head stride below one matrix's rows (heads interleaved inside the token axis) is not
-    // something a 2-D copy can express
-    if (l.kv_heads > 1 && (size_t)l.stride_head * elt < (size_t)(n_in - 1) * row_bytes + (size_t)l.head_dim * elt)
-        return FREQKV_ERR_UNSUPPORTED;
-    cudaError_t e = copy_rows(true, sink, n_in, h2d_bytes);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "host->device copy");
-    st = compress_group(ctx, l, ctx->stage[0], ctx->stage[1], 0, l.batch, n_in, kept_len, sink, variant, stream);
-    if (st != FREQKV_OK) return st;
-    e = copy_rows(false, sink, kept_len, d2h_bytes);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "device->host copy");
+    FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_begin, stream));
+    for (int i = 0; i < 3; ++i) FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[i], ctx->pipe_begin, 0));
+    size_t group = 0;
+    for (int32_t b = 0; b < l.batch; ++b)
+        for (int32_t y0 = 0; y0 < l.layers; y0 += per_group, ++group) {
+            const int32_t ny = std::min(per_group, l.layers - y0);
+            cudaEvent_t copied = ctx->pipe_events[2 * group], compressed = ctx->pipe_events[2 * group + 1];
+            cudaError_t e = copy_rows(true, b, y0, ny, sink, n_in, ctx->pipe[0], h2d_bytes);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "host->device copy");
+            FREQKV_CUDA(ctx, cudaEventRecord(copied, ctx->pipe[0]));
+            FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[1], copied, 0));
+            freqkv_layout sub = l;  // this group's layers of sequence b as a cache of its own
+            sub.batch = 1;
+            sub.layers = ny;
+            const size_t off = ((size_t)b * l.stride_batch + (size_t)y0 * l.stride_layer) * elt;
+            st = compress_group(ctx, sub, static_cast<char*>(ctx->stage[0]) + off, static_cast<char*>(ctx->stage[1]) + off, 0,
+                                1, n_in, kept_len, sink, variant, ctx->pipe[1]);
+            if (st != FREQKV_OK) return st;
+            FREQKV_CUDA(ctx, cudaEventRecord(compressed, ctx->pipe[1]));
+            FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[2], compressed, 0));
+            e = copy_rows(false, b, y0, ny, sink, kept_len, ctx->pipe[2], d2h_bytes);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "device->host copy");
+        }
+    // every copy back is on pipe[2], after the work it depends on: its tail is the end of the call
+    FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_end, ctx->pipe[2]));
+    FREQKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->pipe_end, 0));
     return FREQKV_OK;
 }
 

@@ -232,6 +232,31 @@ def test_gemm_in_place_equals_fresh_copy(ctx):
     assert torch.equal(k, k2) and torch.equal(v, v2)
 
 
+# ---- host-buffer entry point: cache in host memory, copies pipelined with the compression
+@pytest.mark.parametrize("layers,pinned", [(3, True), (20, True), (5, False)])
+def test_compress_host_matches_device_path(ctx, layers, pinned):
+    """Same bits as freqkv_compress on a device copy; rows outside [sink, sink+kept) of the host
+    cache untouched; byte counts are those of the rows moved."""
+    w = small(cap=300, dtype=torch.bfloat16, sink=4, outliers=2, B=2, Ly=layers, H=2)
+    k, v = synth.make_cache(w, "cuda")
+    kh, vh = k.cpu(), v.cpu()
+    if pinned:
+        kh, vh = kh.pin_memory(), vh.pin_memory()
+    kh0, vh0 = kh.clone(), vh.clone()
+    ctx.set_variant(fk.AUTO)
+    new_len, h2d, d2h = ctx.compress_host(kh, vh, 300, 148, 4)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == fk.OK and new_len == 152
+    rows = 2 * 2 * layers * 2  # tensors x batch x layers x heads
+    assert h2d == rows * 296 * 128 * 2 and d2h == rows * 148 * 128 * 2
+    ctx.compress(k, v, 300, 148, 4)
+    assert torch.equal(kh, k.cpu()) and torch.equal(vh, v.cpu())
+    for t, t0 in ((kh, kh0), (vh, vh0)):
+        assert torch.equal(t[..., :4, :], t0[..., :4, :]) and torch.equal(t[..., 152:, :], t0[..., 152:, :])
+    want = oracle.compress_matrix(parity.to_f64(kh0[1, layers - 1, 1, 4:300]), 148)
+    assert parity.rel_l2(parity.to_f64(kh[1, layers - 1, 1, 4:152]), want) < 1e-2
+
+
 # ---- fast-transform variant (power-of-two lengths), in place without scratch
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("n_in,kept,sink", [(128, 64, 0), (256, 128, 4), (512, 256, 0), (1024, 128, 4), (2048, 16, 1),

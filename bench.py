@@ -311,6 +311,50 @@ def run_stream(args, ctx, fk, synth, w, dev, peaks, total_tokens=32768):
             "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": None}
 
 
+def run_attend(args, ctx, fk, synth, name, dev, peaks):
+    """Decode attention of one new token per sequence over full caches (the step after the
+    compression path): one freqkv_attend_decode call per step, layers alternating so that no
+    call finds its rows in L2."""
+    import dataclasses
+
+    B, H, G, cap, base, rho = {"attend_7b": (16, 32, 1, 4096, 10000.0, 0.9), "attend_8b": (8, 8, 4, 8192, 500000.0, 0.95)}[name]
+    layers = 4
+    w = synth.Workload(name, B, layers, H, 128, cap, torch.bfloat16, 4, rho, 2, synth.BASE_SEED + 7)
+    k, v = synth.make_cache(w, dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed + 1)
+    q = torch.randn(B, H * G, 128, generator=gen, device=dev).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    lens = [cap] * B
+    bytes_per_call = 2 * B * H * cap * 128 * 2  # every K and V row of the layer once
+    for i in range(max(args.warmup, 3)):
+        ctx.attend_decode(k, v, i % layers, q, lens, rope_base=base, out=out)
+    torch.cuda.synchronize()
+    ctx.get_timing()
+    ctx.set_timing(True)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(args.steps):
+        ctx.attend_decode(k, v, i % layers, q, lens, rope_base=base, out=out)
+    b.record()
+    torch.cuda.synchronize()
+    n, t_ms, _ = ctx.get_timing()
+    ctx.set_timing(False)
+    ms = a.elapsed_time(b) / args.steps
+    kernel_ms = t_ms / max(n, 1)
+    achieved = bytes_per_call / (kernel_ms * 1e-3) / 1e9
+    return {"metric": "decode attention GB/s of cache read", "value": bytes_per_call / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "batch": B, "kv_heads": H, "q_heads_per_kv": G, "head_dim": 128, "cache_len": cap,
+                       "rope_base": base, "step": "one freqkv_attend_decode call over one layer",
+                       "l2": "%d layers alternate, %.2f GB read per call" % (layers, bytes_per_call / 1e9)},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "peak_kind": "copy, of " + peaks["source"],
+                         "kernel": "attend_partial_kernel + attend_merge_kernel", "kernel_ms": kernel_ms, "traffic": None},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -333,6 +377,15 @@ def main():
     from paper_2505_00570_b200 import binding as fk
     from paper_2505_00570_b200 import synth
 
+    if args.workload in ("attend_7b", "attend_8b"):   # side workload: the step after the compression path
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            ctx = fk.Context(local_rank)
+            print(json.dumps(run_attend(args, ctx, fk, synth, args.workload, torch.device("cuda", local_rank), load_peaks())), flush=True)
+            ctx.close()
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)

@@ -137,6 +137,28 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
                                    int32_t cache_len, int32_t kept_len, int32_t sink, void* cuda_stream,
                                    int64_t* h2d_bytes, int64_t* d2h_bytes);
 
+/* Attention of one newly incoming token per sequence over the bounded cache of one layer
+ * (Section 3.4: the new token attends to the sink tokens, the compressed tokens and the recent
+ * tokens, i.e. to cache rows [0, lens[b]) of its KV head; its own key and value are the last of
+ * those rows, appended before this call).
+ * Position encoding (Section 3.4, last paragraph): keys are cached BEFORE RoPE.  Here cached key
+ * row j is rotated to position j -- its index inside the cache, not inside the original sequence
+ * -- and the query to position lens[b] - 1.  RoPE pairs channel c with channel c + head_dim/2 (the
+ * LLaMA layout) and turns pair c by  position * rope_base^(-2c/head_dim);  rope_base <= 0 switches
+ * it off (plain softmax attention).
+ *   q, out  DEVICE pointers, dense [batch, kv_heads * q_heads_per_kv, head_dim] in the cache dtype;
+ *           query head i uses KV head i / q_heads_per_kv (grouped-query attention); q is given
+ *           before RoPE; out = softmax(scale * q_rot . K_rot^T) V, fp32 arithmetic, rounded once.
+ *   scale   score scale; <= 0 selects 1/sqrt(head_dim).
+ *   lens    HOST array of `batch` cache lengths, each in [1, capacity].
+ * Nothing in the cache is written.  Errors: INVALID_ARG (null pointers, q == out, layer out of
+ * range, a length outside [1, capacity], NaN scale or base), UNSUPPORTED (head_dim != 128,
+ * q_heads_per_kv not 1, 2, 4 or 8, misaligned pointers, layout rules), ALLOC, CUDA.  The first call
+ * with a new rope_base builds a cos/sin table (capacity x head_dim/2 entries) the context keeps. */
+freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v,
+                                   int32_t layer, const void* q, void* out, int32_t q_heads_per_kv, const int32_t* lens,
+                                   float rope_base, float scale, void* cuda_stream);
+
 /* Instrumentation for benchmarks.  With timing enabled every compression records a CUDA event
  * pair on the caller's stream around its transform kernel (the projection / fast-transform
  * launch, not the copy-back or table builders).  freqkv_get_timing waits for the recorded
@@ -185,12 +207,15 @@ freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, void* k, void
 freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream);
 
 /* Host-only argument checks, exactly the ones freqkv_compress / freqkv_append apply before
- * they enqueue anything (they touch no device and need no context): the status those calls
+ * they enqueue anything (they touch no device and need no context; freqkv_check_attend likewise
+ * for freqkv_attend_decode): the status those calls
  * would return for these arguments, FREQKV_OK if they would go ahead. */
 freqkv_status freqkv_check_compress(const freqkv_layout* layout, const void* k, const void* v, int32_t cache_len,
                                     int32_t kept_len, int32_t sink);
 freqkv_status freqkv_check_append(const freqkv_layout* layout, const void* k, const void* v, const void* new_k,
                                   const void* new_v, int32_t n_new, const int32_t* lens);
+freqkv_status freqkv_check_attend(const freqkv_layout* layout, const void* k, const void* v, int32_t layer, const void* q,
+                                  const void* out, int32_t q_heads_per_kv, const int32_t* lens);
 
 /* Text of the most recent CUDA failure or device-status report seen by this context (owned by
  * the context, valid until its next call); "" if none. */

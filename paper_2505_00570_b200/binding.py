@@ -26,7 +26,8 @@ EXPORTS = [
     "freqkv_resolve_variant", "freqkv_plan", "freqkv_compress", "freqkv_compress_ragged",
     "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
-    "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc",
+    "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc", "freqkv_attend_decode",
+    "freqkv_check_attend",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -78,6 +79,9 @@ def lib() -> ctypes.CDLL:
         L.freqkv_set_timing.argtypes = [c_void_p, c_int32]
         L.freqkv_get_timing.argtypes = [c_void_p, POINTER(c_int64), POINTER(ctypes.c_double), POINTER(c_int64)]
         L.freqkv_compress_noalloc.argtypes = [LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
+        L.freqkv_attend_decode.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, I32P,
+                                           ctypes.c_float, ctypes.c_float, c_void_p]
+        L.freqkv_check_attend.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, I32P]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -122,6 +126,11 @@ def check_compress(layout: Layout, k_ptr: int, v_ptr: int, cache_len: int, kept_
 def check_append(layout: Layout, k_ptr: int, v_ptr: int, nk_ptr: int, nv_ptr: int, n_new: int, lens) -> int:
     arr = (c_int32 * len(lens))(*lens)
     return lib().freqkv_check_append(ctypes.byref(layout), k_ptr, v_ptr, nk_ptr, nv_ptr, n_new, arr)
+
+
+def check_attend(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_ptr: int, out_ptr: int, group: int, lens) -> int:
+    arr = (c_int32 * len(lens))(*lens)
+    return lib().freqkv_check_attend(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, arr)
 
 
 def _stream_ptr(stream) -> int:
@@ -229,6 +238,27 @@ class Context:
                                  new_v.data_ptr(), n_new, c_lens, _stream_ptr(stream))
         self._check(st, "freqkv_append")
         return list(c_lens)
+
+    def attend_decode(self, k: torch.Tensor, v: torch.Tensor, layer: int, q: torch.Tensor, lens: list[int],
+                      rope_base: float = 10000.0, scale: float = 0.0, out: torch.Tensor | None = None,
+                      stream=None) -> torch.Tensor:
+        """Attention of one new token per sequence over cache rows [0, lens[b]) of `layer`
+        (keys rotated to their in-cache positions).  ``q``: dense [batch, q_heads, head_dim], cache
+        dtype, before RoPE; q_heads must be a multiple of the cache's kv_heads.  Returns ``out``."""
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        if q.dim() != 3 or not q.is_contiguous() or q.dtype != k.dtype or q.shape[0] != lay.batch or \
+                q.shape[2] != lay.head_dim or q.shape[1] % lay.kv_heads != 0:
+            raise FreqKVError(ERR_INVALID_ARG, "q must be dense [batch, q_heads, head_dim] in the cache dtype")
+        if out is None:
+            out = torch.empty_like(q)
+        c_lens = (c_int32 * lay.batch)(*lens)
+        st = lib().freqkv_attend_decode(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), layer, q.data_ptr(),
+                                        out.data_ptr(), q.shape[1] // lay.kv_heads, c_lens, rope_base, scale,
+                                        _stream_ptr(stream))
+        self._check(st, "freqkv_attend_decode")
+        return out
 
     def compress_host(self, k_host: torch.Tensor, v_host: torch.Tensor, cache_len: int, kept_len: int, sink: int,
                       stream=None) -> tuple[int, int, int]:

@@ -2,6 +2,7 @@
 // All arithmetic of the hot path runs in the kernels this file launches; nothing here touches
 // cache contents on the host.
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -14,6 +15,7 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "fdct.cuh"
+#include "attend.cuh"
 
 using namespace freqkv;
 
@@ -36,6 +38,12 @@ struct freqkv_ctx {
     // host-buffer entry point: device staging caches
     void* stage[2] = {nullptr, nullptr};
     size_t stage_bytes = 0;
+    // decode attention: RoPE table of one base, partial results of the row splits
+    float2* rope_table = nullptr;
+    int32_t rope_rows = 0;
+    double rope_base = 0.0;
+    float* attend_partial = nullptr;
+    size_t attend_partial_bytes = 0;
     cudaStream_t pipe[3] = {nullptr, nullptr, nullptr};  // copy in, compress, copy out
     cudaEvent_t pipe_begin = nullptr, pipe_end = nullptr;
     std::vector<cudaEvent_t> pipe_events;                // per group: copied in, compressed
@@ -429,6 +437,8 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     for (int i = 0; i < 2; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    if (ctx->rope_table) cudaFree(ctx->rope_table);
+    if (ctx->attend_partial) cudaFree(ctx->attend_partial);
     for (int i = 0; i < 3; ++i)
         if (ctx->pipe[i]) cudaStreamDestroy(ctx->pipe[i]);
     if (ctx->pipe_begin) cudaEventDestroy(ctx->pipe_begin);
@@ -685,6 +695,78 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
     // every copy back is on pipe[2], after the work it depends on: its tail is the end of the call
     FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_end, ctx->pipe[2]));
     FREQKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->pipe_end, 0));
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_check_attend(const freqkv_layout* layout, const void* k, const void* v, int32_t layer, const void* q,
+                                  const void* out, int32_t q_heads_per_kv, const int32_t* lens)
+{
+    if (!lens) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    st = check_tensors(*layout, k, v);
+    if (st != FREQKV_OK) return st;
+    if (!q || !out || q == out) return FREQKV_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return FREQKV_ERR_UNSUPPORTED;
+    if (layer < 0 || layer >= layout->layers || q_heads_per_kv < 1) return FREQKV_ERR_INVALID_ARG;
+    if (!attend_supported(layout->head_dim, q_heads_per_kv)) return FREQKV_ERR_UNSUPPORTED;
+    for (int32_t b = 0; b < layout->batch; ++b)
+        if (lens[b] < 1 || lens[b] > layout->capacity) return FREQKV_ERR_INVALID_ARG;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v, int32_t layer,
+                                   const void* q, void* out, int32_t q_heads_per_kv, const int32_t* lens, float rope_base,
+                                   float scale, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    const freqkv_status st = freqkv_check_attend(layout, k, v, layer, q, out, q_heads_per_kv, lens);
+    if (st != FREQKV_OK) return st;
+    if (!(scale == scale) || !(rope_base == rope_base)) return FREQKV_ERR_INVALID_ARG;  // NaN
+    const freqkv_layout& l = *layout;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (scale <= 0.f) scale = 1.0f / sqrtf((float)l.head_dim);
+    int32_t max_len = 0;
+    for (int32_t b = 0; b < l.batch; ++b) max_len = std::max(max_len, lens[b]);
+    const float2* table = nullptr;
+    if (rope_base > 0.f) {
+        if (!ctx->rope_table || ctx->rope_rows < l.capacity || ctx->rope_base != (double)rope_base) {
+            if (ctx->rope_table) {
+                FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // an enqueued launch may still read the old table
+                cudaFree(ctx->rope_table);
+                ctx->rope_table = nullptr;
+            }
+            const int32_t rows = std::max(l.capacity, 2);
+            FREQKV_CUDA(ctx, cudaMalloc(&ctx->rope_table, (size_t)rows * 64 * sizeof(float2)));
+            const cudaError_t e = launch_rope_table(ctx->rope_table, rows, (double)rope_base, stream);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "rope_table");
+            ctx->rope_rows = rows;
+            ctx->rope_base = (double)rope_base;
+            ctx->kernels_launched += 1;
+        }
+        table = ctx->rope_table;
+    }
+    const int32_t splits = attend_splits(l.batch, l.kv_heads, max_len, q_heads_per_kv, ctx->sm_count);
+    const size_t need = attend_partial_bytes(splits, l.batch, l.kv_heads * q_heads_per_kv);
+    if (need > ctx->attend_partial_bytes) {
+        if (ctx->attend_partial) {
+            FREQKV_CUDA(ctx, cudaDeviceSynchronize());
+            cudaFree(ctx->attend_partial);
+            ctx->attend_partial = nullptr;
+            ctx->attend_partial_bytes = 0;
+        }
+        FREQKV_CUDA(ctx, cudaMalloc(&ctx->attend_partial, need));
+        ctx->attend_partial_bytes = need;
+    }
+    cudaError_t e;
+    {
+        TransformTimer timer(ctx, stream);
+        e = launch_attend(l, k, v, layer, q, out, q_heads_per_kv, lens, table, scale, splits, ctx->attend_partial, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "attend");
+    ctx->kernels_launched += 1 + (l.batch + ATTEND_MAX_BATCH - 1) / ATTEND_MAX_BATCH;
     return FREQKV_OK;
 }
 

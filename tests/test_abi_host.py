@@ -124,6 +124,23 @@ def test_check_append():
     assert fk.check_append(L, K, V, NK, NV, -1, [0, 0]) == fk.ERR_INVALID_ARG
 
 
+def test_check_attend():
+    L = lay(cap=64, B=2)
+    Q, O = 0x30000000, 0x40000000
+    assert fk.check_attend(L, K, V, 0, Q, O, 1, [1, 64]) == fk.OK
+    assert fk.check_attend(L, K, V, 0, Q, O, 4, [10, 20]) == fk.OK
+    assert fk.check_attend(L, K, V, 0, Q, O, 3, [10, 20]) == fk.ERR_UNSUPPORTED      # group size not 1, 2, 4, 8
+    assert fk.check_attend(L, K, V, 0, Q, O, 0, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, 0, Q, O, 1, [0, 20]) == fk.ERR_INVALID_ARG       # an empty cache has nothing to attend to
+    assert fk.check_attend(L, K, V, 0, Q, O, 1, [10, 65]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, L.layers, Q, O, 1, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, -1, Q, O, 1, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, 0, Q, Q, 1, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, 0, 0, O, 1, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend(L, K, V, 0, Q + 2, O, 1, [10, 20]) == fk.ERR_UNSUPPORTED
+    assert fk.check_attend(lay(hd=64), K, V, 0, Q, O, 1, [10]) == fk.ERR_UNSUPPORTED
+
+
 def test_null_context_is_rejected():
     L = lay()
     lib = fk.lib()

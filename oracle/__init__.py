@@ -105,6 +105,25 @@ def compress_matrix(x, kept_len: int) -> np.ndarray:
     return y
 
 
+def compress_band_matrix(x, kept_len: int, first: int) -> np.ndarray:
+    """The ablation of Appendix "Retaining High/Low-Frequency Components": keep the ``kept_len``
+    DCT components ``first .. first + kept_len - 1`` instead of the lowest ones, then the same
+    L-point inverse and rescale:  sqrt(L/N) * IDCT_L(DCT_N(x)[first : first + L]).
+    ``first = 0`` is ``compress_matrix``; ``first = N - L`` retains the highest frequencies.
+    (The paper does not say where the retained components go in the inverse transform; they
+    take positions 0 .. L-1 here, the only choice that keeps the output length L.)"""
+    x = _as_matrix(x)
+    N, d = x.shape
+    L, t0 = int(kept_len), int(first)
+    if L < 0 or t0 < 0 or t0 + L > N:
+        raise ValueError("need 0 <= first and first + kept_len <= N")
+    if L == 0:
+        return np.empty((0, d))
+    z = dct2(x)                      # all N components (Appendix A, DCT-II)
+    kept = np.ascontiguousarray(z[t0:t0 + L])
+    return np.sqrt(L / N) * idct(kept)
+
+
 def compress_cache(cache, cache_len: int, kept_len: int, sink: int) -> tuple[np.ndarray, int]:
     """One compression of every matrix of a cache (Sections 3.3-3.4).
 

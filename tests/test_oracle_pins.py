@@ -229,3 +229,45 @@ def test_ar1_energy_is_low_frequency():
     frac = (y ** 2).mean() / 1.0
     expected = (2 / math.pi) * math.atan((1 + w.rho) / (1 - w.rho))  # AR(1) low-half energy
     assert abs(frac - expected) < 0.05
+
+
+# ---- retaining another band of components (the high/low-frequency ablation)
+@pytest.mark.parametrize("N,L", [(8, 4), (31, 15), (128, 64), (257, 100)])
+def test_band_zero_offset_is_the_low_pass_compression(N, L):
+    x = rng(N + L).standard_normal((N, 3))
+    assert rel(oracle.compress_band_matrix(x, L, 0), oracle.compress_matrix(x, L)) < TOL
+
+
+@pytest.mark.parametrize("N,L,t0", [(12, 6, 6), (12, 5, 3), (64, 32, 32), (100, 25, 60), (31, 15, 16)])
+def test_band_single_cosine_is_shifted_down_and_resampled(N, L, t0):
+    """x_n = cos(pi k (2n+1)/(2N)) has the single DCT component k; retained in the band it becomes
+    component k - t0 of the L-point inverse: y_m = cos(pi (k - t0)(2m+1)/(2L)) (times 1/sqrt 2 when it
+    lands on component 0, whose weight differs); outside the band the output is zero."""
+    n, m = np.arange(N), np.arange(L)
+    for k in {t0, t0 + 1, t0 + L - 1, max(0, t0 - 1), min(N - 1, t0 + L)} - {0}:
+        x = np.cos(np.pi * k * (2 * n + 1) / (2 * N))[:, None]
+        y = oracle.compress_band_matrix(x, L, t0)[:, 0]
+        if t0 <= k < t0 + L:
+            want = np.cos(np.pi * (k - t0) * (2 * m + 1) / (2 * L)) * (1 / math.sqrt(2) if k == t0 else 1.0)
+        else:
+            want = np.zeros(L)
+        assert np.max(np.abs(y - want)) < 1e-11
+
+
+@pytest.mark.parametrize("N,L,t0", [(64, 32, 32), (100, 30, 11), (257, 100, 157)])
+def test_band_parseval_and_linearity(N, L, t0):
+    r = rng(N * 7 + t0)
+    x, x2 = r.standard_normal((N, 4)), r.standard_normal((N, 4))
+    z = scipy.fft.dct(x, type=2, norm="ortho", axis=0)
+    y = oracle.compress_band_matrix(x, L, t0)
+    assert abs(np.sum(y * y) - (L / N) * np.sum(z[t0:t0 + L] ** 2)) < 1e-10 * np.sum(x * x)
+    want = math.sqrt(L / N) * scipy.fft.idct(z[t0:t0 + L], type=2, norm="ortho", axis=0)   # library pipeline
+    assert rel(y, want) < TOL
+    assert rel(oracle.compress_band_matrix(2 * x - 3 * x2, L, t0), 2 * y - 3 * oracle.compress_band_matrix(x2, L, t0)) < TOL
+
+
+def test_band_low_plus_high_halves_carry_all_the_energy():
+    N = 64
+    x = rng(5).standard_normal((N, 2))
+    lo, hi = oracle.compress_band_matrix(x, 32, 0), oracle.compress_band_matrix(x, 32, 32)
+    assert abs(np.sum(lo * lo) + np.sum(hi * hi) - 0.5 * np.sum(x * x)) < 1e-10

@@ -365,6 +365,9 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "gemm", "fdct", "simt"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--retain", type=float, default=0.5, help="retaining ratio gamma: kept_len = floor(gamma * (cache_len - sink))")
+    ap.add_argument("--high-frequencies", action="store_true",
+                    help="retain the highest kept_len DCT components instead of the lowest (the paper's ablation)")
     ap.add_argument("--layers", type=int, default=0, help="shrink the workload to this many layers (profiling only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -402,7 +405,8 @@ def main():
 
         w = dataclasses.replace(w, layers=args.layers)
     cache_len, sink = w.capacity, w.sink
-    kept = w.kept_len(cache_len)
+    kept = w.kept_len(cache_len, args.retain)
+    first = cache_len - sink - kept if args.high_frequencies else 0
     n_new = cache_len - sink - kept
     nums = workload_numbers(w, cache_len, kept, sink)
 
@@ -434,7 +438,7 @@ def main():
         except fk.FreqKVError as err:
             if err.status != fk.ERR_CAPACITY:
                 raise
-        new_len = ctx.compress(k, v, cache_len, kept, sink)
+        new_len = ctx.compress_band(k, v, cache_len, kept, sink, first) if first else ctx.compress(k, v, cache_len, kept, sink)
         return ctx.append(k, v, nk, nv, [new_len] * w.batch)
 
     for _ in range(args.warmup):
@@ -481,7 +485,8 @@ def main():
         return a.elapsed_time(b) / reps
 
     reps = max(3, min(args.steps, 20))
-    compress_ms = timed(lambda: ctx.compress(k, v, cache_len, kept, sink), reps)
+    compress_ms = timed(lambda: ctx.compress_band(k, v, cache_len, kept, sink, first) if first
+                        else ctx.compress(k, v, cache_len, kept, sink), reps)
     append_ms = timed(lambda: ctx.append(k, v, nk, nv, [sink + kept] * w.batch), reps)
 
     # ---- roofline of the dominant kernel (the transform launch)
@@ -541,7 +546,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "batch": w.batch, "layers": w.layers, "kv_heads": w.kv_heads,
                        "head_dim": w.head_dim, "capacity": w.capacity, "cache_len": cache_len, "sink": sink,
-                       "kept_len": kept, "appended_rows_per_step": n_new, "variant": chosen_name,
+                       "kept_len": kept, "first_component": first, "appended_rows_per_step": n_new, "variant": chosen_name,
                        "l2": "inputs larger than L2 (%.2f GB of cache per step)" % (nums["cache_in_bytes"] / 1e9),
                        "parallelism": "replicas only" if n_gpus > 1 else "single GPU",
                        "step": "refused append (lazy trigger) + compress K,V in place + append chunk"},

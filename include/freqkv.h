@@ -105,6 +105,18 @@ freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_
 freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
                               int32_t kept_len, int32_t sink, void* cuda_stream);
 
+/* The same compression with another band of components retained (the paper's ablation
+ * "Retaining High/Low-Frequency Components"): components first_component .. first_component +
+ * kept_len - 1 of the N-point DCT-II are kept instead of the lowest kept_len,
+ *     y = sqrt(L/N) * IDCT_L(z[first_component : first_component + L]),
+ * the retained components taking positions 0 .. L-1 of the L-point inverse (the paper does not say
+ * where they go; this keeps the output length L).  first_component = 0 is freqkv_compress;
+ * first_component = N - L retains the highest frequencies.  Same rows written, same errors, plus
+ * INVALID_ARG when first_component < 0 or first_component + kept_len > N.  The fast-transform
+ * variant does not take first_component != 0 (UNSUPPORTED when forced; AUTO uses another variant). */
+freqkv_status freqkv_compress_band(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
+                                   int32_t kept_len, int32_t sink, int32_t first_component, void* cuda_stream);
+
 /* Ragged form: sequence b holds lens[b] rows and is compressed to sink + kept_len[b] rows,
  * each sequence with the transform of its own length (same definition as above with
  * N = lens[b] - sink, L = kept_len[b]).  `lens` and `kept_len` are host arrays of

@@ -27,7 +27,7 @@ EXPORTS = [
     "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
     "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc", "freqkv_attend_decode",
-    "freqkv_check_attend",
+    "freqkv_check_attend", "freqkv_compress_band",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.freqkv_resolve_variant.argtypes = [c_void_p, LP, c_int32, c_int32, I32P]
         L.freqkv_plan.argtypes = [c_void_p, c_int32, c_int32, c_int, c_int, c_void_p]
         L.freqkv_compress.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
+        L.freqkv_compress_band.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p]
         L.freqkv_compress_ragged.argtypes = [c_void_p, LP, c_void_p, c_void_p, I32P, I32P, c_int32, c_void_p]
         L.freqkv_append.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P, c_void_p]
         L.freqkv_last_device_status.argtypes = [c_void_p, c_void_p]
@@ -206,6 +207,18 @@ class Context:
         st = lib().freqkv_compress(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), cache_len, kept_len, sink,
                                    _stream_ptr(stream))
         self._check(st, "freqkv_compress")
+        return sink + kept_len
+
+    def compress_band(self, k: torch.Tensor, v: torch.Tensor, cache_len: int, kept_len: int, sink: int,
+                      first_component: int, stream=None) -> int:
+        """Like ``compress`` but keeping DCT components ``first_component .. first_component +
+        kept_len - 1`` (the high/low-frequency ablation).  Returns the new cache length."""
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        st = lib().freqkv_compress_band(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), cache_len, kept_len, sink,
+                                        first_component, _stream_ptr(stream))
+        self._check(st, "freqkv_compress_band")
         return sink + kept_len
 
     def compress_ragged(self, k: torch.Tensor, v: torch.Tensor, lens: list[int], kept_len: list[int], sink: int,

@@ -9,6 +9,7 @@
 #include <map>
 #include <new>
 #include <string>
+#include <tuple>
 #include <utility>
 #include <vector>
 
@@ -23,7 +24,7 @@ struct freqkv_ctx {
     int device = 0;
     int sm_count = 0;
     freqkv_variant forced = FREQKV_AUTO;
-    std::map<std::pair<int32_t, int32_t>, Basis> bases;
+    std::map<std::tuple<int32_t, int32_t, int32_t>, Basis> bases;  // (n_in, n_keep, first retained component)
     std::map<std::pair<int32_t, int32_t>, FdctPlan> fdct_plans;
     size_t basis_bytes = 0;
     void* scratch = nullptr;
@@ -187,10 +188,10 @@ void free_bases(freqkv_ctx* ctx)
 
 // Projection basis for (n_in, n_keep) holding at least the requested forms: the full fp32 matrix
 // (CUDA-core path) and/or the folded bf16 pair Pe, Po (tensor-core path).
-freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need_f32, bool need_fold,
+freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t first, bool need_f32, bool need_fold,
                         cudaStream_t stream, Basis* out)
 {
-    const auto key = std::make_pair(n_in, n_keep);
+    const auto key = std::make_tuple(n_in, n_keep, first);
     Basis b;
     auto it = ctx->bases.find(key);
     if (it != ctx->bases.end()) b = it->second;
@@ -199,6 +200,7 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need
         auto shape = [&](Basis& x) {
             x.n_in = n_in;
             x.n_keep = n_keep;
+            x.first = first;
             x.ld = (n_in + 63) / 64 * 64;
             x.rows_pad = (n_keep + 63) / 64 * 64;
             x.fold_ld = ((n_in + 1) / 2 + 63) / 64 * 64;
@@ -226,11 +228,11 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, bool need
         }
         cudaError_t e = cudaSuccess;
         if (pf) {
-            e = launch_build_basis(pf, nullptr, n_in, n_keep, b.ld, b.rows_pad, stream);
+            e = launch_build_basis(pf, nullptr, n_in, n_keep, first, b.ld, b.rows_pad, stream);
             ctx->kernels_launched += 1;
         }
         if (e == cudaSuccess && pb) {
-            e = launch_build_folded_basis(pb, n_in, n_keep, b.fold_ld, b.fold_rows_pad, stream);
+            e = launch_build_folded_basis(pb, n_in, n_keep, first, b.fold_ld, b.fold_rows_pad, stream);
             ctx->kernels_launched += 1;
         }
         if (e != cudaSuccess) {
@@ -297,7 +299,7 @@ struct TransformTimer {
 // Compress `count` sequences starting at batch0, all with the same (n_in, n_keep).
 freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, void* v, int32_t batch0,
                              int32_t batch_count, int32_t n_in, int32_t n_keep, int32_t sink, int32_t variant,
-                             cudaStream_t stream)
+                             cudaStream_t stream, int32_t first = 0)
 {
     const CacheView view = make_view(l, k, v, batch0, batch_count);
     const int32_t n_mat = 2 * view.mats_per_tensor;
@@ -325,7 +327,7 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
 
     Basis basis;
     const bool gemm = variant == FREQKV_GEMM;
-    freqkv_status st = get_basis(ctx, n_in, n_keep, !gemm, gemm, stream, &basis);
+    freqkv_status st = get_basis(ctx, n_in, n_keep, first, !gemm, gemm, stream, &basis);
     if (st != FREQKV_OK) return st;
 
     if (gemm) {
@@ -496,7 +498,7 @@ freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_
     Basis b;
     const bool gemm = variant == FREQKV_GEMM;
     const bool both = variant == FREQKV_AUTO;
-    return get_basis(ctx, n_in, n_keep, !gemm || both, (gemm || both) && dtype == FREQKV_BF16, stream, &b);
+    return get_basis(ctx, n_in, n_keep, 0, !gemm || both, (gemm || both) && dtype == FREQKV_BF16, stream, &b);
 }
 
 freqkv_status freqkv_check_compress(const freqkv_layout* layout, const void* k, const void* v, int32_t cache_len,
@@ -541,6 +543,27 @@ freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void
     if (!g.ok) return FREQKV_ERR_CUDA;
     return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
                           static_cast<cudaStream_t>(cuda_stream));
+}
+
+freqkv_status freqkv_compress_band(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
+                                   int32_t kept_len, int32_t sink, int32_t first_component, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = freqkv_check_compress(layout, k, v, cache_len, kept_len, sink);
+    if (st != FREQKV_OK) return st;
+    const int32_t n_in = cache_len - sink;
+    if (first_component < 0 || (int64_t)first_component + kept_len > n_in) return FREQKV_ERR_INVALID_ARG;
+    if (n_in == 0 || kept_len == 0 || kept_len == n_in) return FREQKV_OK;  // nothing to rewrite (a full band is the identity)
+    int32_t variant = resolve(ctx, *layout, n_in, kept_len);
+    if (variant == FREQKV_FDCT && first_component != 0) {  // the fast transform keeps the lowest components only
+        if (ctx->forced == FREQKV_FDCT) return FREQKV_ERR_UNSUPPORTED;
+        variant = FREQKV_SIMT;
+    }
+    if (variant < 0) return FREQKV_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
+                          static_cast<cudaStream_t>(cuda_stream), first_component);
 }
 
 freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t* lens,

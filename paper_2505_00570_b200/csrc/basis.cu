@@ -26,18 +26,51 @@ __device__ inline double dirichlet(int64_t a, int64_t L, int64_t LN4)
     return sinpi((double)r / (double)LN4) / sinpi((double)a / (double)LN4);
 }
 
+// Retaining components t0 .. t0 + L - 1 instead of the lowest L (the paper's high/low-frequency
+// ablation; t0 >= 1 here).  With A = pi (2m+1) / (2L), B = pi (2n+1) / (2N) the orthonormal weights
+// give  P[m][n] = (sqrt 2 / N) [ cos(B t0) + sqrt 2 * sum_{t'=1}^{L-1} cos(A t') cos(B (t0 + t')) ],
+// and each of the two cosine series the product splits into sums in closed form:
+//   sum_{t'=1}^{L-1} cos(theta t' + phi) = sin((L-1) theta / 2) / sin(theta / 2) * cos(L theta / 2 + phi),
+// (L - 1) cos(phi) at theta = 0.  All phases are integer multiples of pi / (4LN) and are reduced
+// exactly modulo 8LN before sinpi / cospi.
+__device__ inline double cos_units(int64_t k, int64_t LN4)
+{
+    const int64_t period = 2 * LN4;
+    k = ((k % period) + period) % period;
+    return cospi((double)k / (double)LN4);
+}
+__device__ inline double sin_units(int64_t k, int64_t LN4)
+{
+    const int64_t period = 2 * LN4;
+    k = ((k % period) + period) % period;
+    return sinpi((double)k / (double)LN4);
+}
+__device__ inline double cosine_series(int64_t a, int64_t phi, int64_t L, int64_t LN4)
+{
+    if (a == 0) return (double)(L - 1) * cos_units(phi, LN4);
+    return sin_units((L - 1) * a, LN4) / sin_units(a, LN4) * cos_units(L * a + phi, LN4);
+}
+
+// P[m][n] of the map that keeps components t0 .. t0 + L - 1 of an N-point signal.
+__device__ inline double basis_entry(int64_t m, int64_t n, int64_t N, int64_t L, int64_t t0)
+{
+    const int64_t LN4 = 4 * L * N;
+    const int64_t u = (2 * m + 1) * N, w = (2 * n + 1) * L;
+    if (t0 == 0) return (dirichlet(u + w, L, LN4) + dirichlet(u - w, L, LN4)) / (double)(2 * N);
+    const int64_t phi = (2 * n + 1) * t0 * 2 * L;
+    const double series = 0.5 * (cosine_series(u + w, phi, L, LN4) + cosine_series(u - w, -phi, L, LN4));
+    return 1.4142135623730951 / (double)N * (cos_units(phi, LN4) + 1.4142135623730951 * series);
+}
+
 __global__ void build_basis_kernel(float* __restrict__ p_f32, __nv_bfloat16* __restrict__ p_bf16, int32_t n_in,
-                                   int32_t n_keep, int32_t ld, int32_t rows_pad)
+                                   int32_t n_keep, int32_t first, int32_t ld, int32_t rows_pad)
 {
     const int64_t total = (int64_t)rows_pad * ld;
-    const int64_t N = n_in, L = n_keep, LN4 = 4 * L * N;
+    const int64_t N = n_in, L = n_keep;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t m = i / ld, n = i % ld;
         double p = 0.0;
-        if (m < L && n < N) {
-            const int64_t u = (2 * m + 1) * N, w = (2 * n + 1) * L;
-            p = (dirichlet(u + w, L, LN4) + dirichlet(u - w, L, LN4)) / (double)(2 * N);
-        }
+        if (m < L && n < N) p = basis_entry(m, n, N, L, first);
         if (p_f32) p_f32[i] = (float)p;
         if (p_bf16) p_bf16[i] = __double2bfloat16(p);
     }
@@ -50,19 +83,20 @@ __global__ void build_basis_kernel(float* __restrict__ p_f32, __nv_bfloat16* __r
 // Only m < ceil(L/2), n < ceil(N/2) are stored: plane 0 = Pe, plane 1 = Po, each rows_pad x ld,
 // zero padded.  For odd N the middle column of Po is zero and that of Pe is P itself, for odd L the
 // middle row of Po is zero: the formulas above give exactly that.
-__global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32_t n_in, int32_t n_keep, int32_t ld,
-                                          int32_t rows_pad)
+// When a band starting at an odd component t0 is retained, the parity of the inverse's index t'
+// is opposite to that of t = t0 + t': Pe is then antisymmetric and Po symmetric under m -> L-1-m,
+// which only changes a sign in the tensor-core kernel's epilogue.
+__global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32_t n_in, int32_t n_keep, int32_t first,
+                                          int32_t ld, int32_t rows_pad)
 {
     const int64_t plane = (int64_t)rows_pad * ld;
-    const int64_t N = n_in, L = n_keep, LN4 = 4 * L * N;
+    const int64_t N = n_in, L = n_keep;
     const int64_t Nh = (N + 1) / 2, Lh = (L + 1) / 2;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t m = i / ld, n = i % ld;
         double pe = 0.0, po = 0.0;
         if (m < Lh && n < Nh) {
-            const int64_t u = (2 * m + 1) * N, w = (2 * n + 1) * L, wr = (2 * (N - 1 - n) + 1) * L;
-            const double a = (dirichlet(u + w, L, LN4) + dirichlet(u - w, L, LN4)) / (double)(2 * N);
-            const double b = (dirichlet(u + wr, L, LN4) + dirichlet(u - wr, L, LN4)) / (double)(2 * N);
+            const double a = basis_entry(m, n, N, L, first), b = basis_entry(m, N - 1 - n, N, L, first);
             pe = 0.5 * (a + b);
             po = 0.5 * (a - b);
         }
@@ -73,27 +107,27 @@ __global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32
 
 }  // namespace
 
-cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
-                                      cudaStream_t stream)
+cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t first, int32_t ld,
+                                      int32_t rows_pad, cudaStream_t stream)
 {
     const int64_t total = (int64_t)rows_pad * ld;
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (blocks < 1) blocks = 1;
-    build_folded_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(out, n_in, n_keep, ld, rows_pad);
+    build_folded_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(out, n_in, n_keep, first, ld, rows_pad);
     return cudaGetLastError();
 }
 
-cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
-                               int32_t rows_pad, cudaStream_t stream)
+cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t first,
+                               int32_t ld, int32_t rows_pad, cudaStream_t stream)
 {
     const int64_t total = (int64_t)rows_pad * ld;
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (blocks < 1) blocks = 1;
-    build_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(p_f32, p_bf16, n_in, n_keep, ld, rows_pad);
+    build_basis_kernel<<<(unsigned)blocks, threads, 0, stream>>>(p_f32, p_bf16, n_in, n_keep, first, ld, rows_pad);
     return cudaGetLastError();
 }
 

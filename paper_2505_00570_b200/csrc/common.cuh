@@ -38,6 +38,7 @@ __host__ __device__ inline void* tensor_base(const CacheView& v, int32_t tensor)
 struct Basis {
     float* f32 = nullptr;  // SIMT path
     int32_t n_in = 0, n_keep = 0, ld = 0, rows_pad = 0;
+    int32_t first = 0;     // first retained DCT component (0 = the lowest n_keep components)
     // Tensor-core path: the even-frequency and odd-frequency parts Pe, Po of P restricted to
     // m < ceil(n_keep/2), n < ceil(n_in/2), bf16, two planes of fold_rows_pad x fold_ld (see basis.cu).
     __nv_bfloat16* fold = nullptr;
@@ -47,12 +48,13 @@ struct Basis {
 // ---- kernel launchers (each returns the cudaError_t of its launch) ----
 
 // P[m][n] for m < n_keep, n < n_in from the closed form; zero padding elsewhere.
-cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t ld,
-                               int32_t rows_pad, cudaStream_t stream);
+// (`first` = index of the first retained DCT component; 0 for the method's low-pass compression)
+cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t first,
+                               int32_t ld, int32_t rows_pad, cudaStream_t stream);
 
 // Pe and Po of the folded basis (two planes of rows_pad x ld), zero padding elsewhere.
-cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
-                                      cudaStream_t stream);
+cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t first, int32_t ld,
+                                      int32_t rows_pad, cudaStream_t stream);
 
 // scratch[i - first][m][c] = sum_n P[m][n] * X_i[sink + n][c] for matrices first .. first+count-1.
 cudaError_t launch_project_simt(const CacheView& view, int32_t dtype, int32_t first, int32_t count, const Basis& basis,

@@ -71,6 +71,7 @@ struct GemmParams {
     int32_t pair0, pair_count;  // (batch, layer, kv_head) triples covered by this launch
     int32_t m_pairs, k_steps;   // tiles of 256 folded rows per (batch, layer, kv_head); slices per phase
     int32_t sink;
+    int32_t mirror_sign;        // +1: y[L-1-m] = s - d;  -1: y[L-1-m] = d - s (a retained band that starts at an odd component)
     int32_t* status;
 };
 
@@ -456,6 +457,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             const int32_t m = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
             const int32_t mr = prm.n_keep - 1 - m;
             const bool row_ok = m < prm.rows_half;
+            const float sgn = (float)prm.mirror_sign;
             __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
                                  matrix_offset(view, prm.pair0 + pair_local) + (int64_t)prm.sink * view.stride_token;
             uint4* out_p = reinterpret_cast<uint4*>(mat + (int64_t)m * view.stride_token);
@@ -472,7 +474,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         const float s0 = __uint_as_float(s[c * 16 + 2 * j]), s1 = __uint_as_float(s[c * 16 + 2 * j + 1]);
                         const float d0 = __uint_as_float(d[2 * j]), d1 = __uint_as_float(d[2 * j + 1]);
                         p[j] = pack_bf16(s0 + d0, s1 + d1);
-                        q[j] = pack_bf16(s0 - d0, s1 - d1);
+                        q[j] = pack_bf16(sgn * (s0 - d0), sgn * (s1 - d1));
                     }
                     out_p[2 * c] = make_uint4(p[0], p[1], p[2], p[3]);
                     out_p[2 * c + 1] = make_uint4(p[4], p[5], p[6], p[7]);
@@ -646,6 +648,7 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         prm.m_pairs = m_pairs;
         prm.k_steps = (n_half + BK - 1) / BK;
         prm.sink = sink;
+        prm.mirror_sign = (basis.first & 1) ? -1 : 1;
         prm.status = status_dev;
         const int32_t tiles = job.pair_count * m_pairs;
         const int clusters = std::min<int32_t>(tiles, state->max_clusters);

@@ -114,7 +114,7 @@ extern "C" freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, vo
         const int32_t chunk = (int32_t)std::min<size_t>(kStagingBytes / per_matrix, (size_t)n_mat);
         // The basis array keeps whatever the previous call left: the builder rewrites the whole
         // padded rectangle this call reads, zeros included.
-        cudaError_t e = launch_build_basis(arrays.basis, nullptr, n_in, kept_len, basis.ld, basis.rows_pad, stream);
+        cudaError_t e = launch_build_basis(arrays.basis, nullptr, n_in, kept_len, 0, basis.ld, basis.rows_pad, stream);
         for (int32_t first = 0; e == cudaSuccess && first < n_mat; first += chunk) {
             const int32_t count = std::min(chunk, n_mat - first);
             e = launch_project_simt(view, layout->dtype, first, count, basis, sink, arrays.staging, stream);

@@ -232,6 +232,46 @@ def test_gemm_in_place_equals_fresh_copy(ctx):
     assert torch.equal(k, k2) and torch.equal(v, v2)
 
 
+# ---- other retention patterns: retaining ratios 0.25 / 0.75 / 1 %, and another band of components
+@pytest.mark.parametrize("n_in,kept", [(4092, 1023), (4092, 3069), (4092, 40), (1000, 10)])
+def test_other_retaining_ratios_gemm(ctx, n_in, kept):
+    w = small(cap=n_in + 4, dtype=torch.bfloat16, sink=4, outliers=2, Ly=1, H=2)
+    parity.check_compress(ctx, w, n_in + 4, kept, 4, fk.GEMM)
+
+
+@pytest.mark.parametrize("variant,dtype", [(fk.GEMM, torch.bfloat16), (fk.SIMT, torch.float32), (fk.SIMT, torch.bfloat16)])
+@pytest.mark.parametrize("n_in,kept,first", [(300, 150, 150), (300, 150, 75), (301, 150, 151), (257, 101, 33),
+                                             (1024, 512, 512), (64, 63, 1), (700, 350, 0)])
+def test_band_retention(ctx, variant, dtype, n_in, kept, first):
+    """Components first .. first+kept-1 retained (first = n_in - kept: the highest frequencies);
+    even and odd `first` take different signs in the tensor-core epilogue."""
+    w = small(cap=n_in + 7, dtype=dtype, sink=4, outliers=2 if dtype == torch.bfloat16 else 0, Ly=2, H=2)
+    if first == 0:
+        parity.check_compress(ctx, w, n_in + 4, kept, 4, variant)
+    else:
+        parity.check_compress(ctx, w, n_in + 4, kept, 4, variant, first=first)
+
+
+def test_band_config2_shape_high_frequencies(ctx):
+    w = dataclasses.replace(synth.WORKLOADS["llama2_7b"], layers=1, kv_heads=4)
+    parity.check_compress(ctx, w, 4096, 2046, 4, fk.AUTO, sample=4, first=2046)
+
+
+def test_band_invalid_and_fast_transform(ctx):
+    k = torch.zeros(1, 1, 1, 600, 128, device="cuda", dtype=torch.bfloat16)
+    v = torch.zeros_like(k)
+    ctx.set_variant(fk.AUTO)
+    for first in (-1, 257):
+        with pytest.raises(fk.FreqKVError) as e:
+            ctx.compress_band(k, v, 516, 256, 4, first)
+        assert e.value.status == fk.ERR_INVALID_ARG
+    ctx.set_variant(fk.FDCT)
+    with pytest.raises(fk.FreqKVError) as e:
+        ctx.compress_band(k, v, 516, 256, 4, 256)
+    assert e.value.status == fk.ERR_UNSUPPORTED
+    ctx.set_variant(fk.AUTO)
+
+
 # ---- host-buffer entry point: cache in host memory, copies pipelined with the compression
 @pytest.mark.parametrize("layers,pinned", [(3, True), (20, True), (5, False)])
 def test_compress_host_matches_device_path(ctx, layers, pinned):

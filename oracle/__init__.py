@@ -124,6 +124,22 @@ def compress_band_matrix(x, kept_len: int, first: int) -> np.ndarray:
     return np.sqrt(L / N) * idct(kept)
 
 
+def power_spectrum(states) -> np.ndarray:
+    """Average power spectrum along the token axis (Section 3.1, the analysis behind the
+    paper's power-spectrum figures): every channel of every ``[N, d]`` matrix in ``states``
+    (``[..., N, d]``; the leading axes are samples) is transformed with the orthonormal DCT-II
+    of Appendix A and the squared components are averaged over samples and channels.
+    Returns ``[N]``.  ("Power" is read as the squared amplitude of a component.)"""
+    a = np.asarray(states, dtype=np.float64)
+    N, d = a.shape[-2], a.shape[-1]
+    flat = a.reshape(-1, N, d)
+    total = np.zeros(N)
+    for x in flat:
+        z = dct2(x)
+        total += np.sum(z * z, axis=1)
+    return total / (flat.shape[0] * d)
+
+
 def compress_cache(cache, cache_len: int, kept_len: int, sink: int) -> tuple[np.ndarray, int]:
     """One compression of every matrix of a cache (Sections 3.3-3.4).
 

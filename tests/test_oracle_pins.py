@@ -271,3 +271,36 @@ def test_band_low_plus_high_halves_carry_all_the_energy():
     x = rng(5).standard_normal((N, 2))
     lo, hi = oracle.compress_band_matrix(x, 32, 0), oracle.compress_band_matrix(x, 32, 32)
     assert abs(np.sum(lo * lo) + np.sum(hi * hi) - 0.5 * np.sum(x * x)) < 1e-10
+
+
+# ---- average power spectrum (Section 3.1)
+def test_power_spectrum_parseval_constant_and_single_cosine():
+    N, d = 96, 5
+    x = rng(21).standard_normal((3, N, d))
+    p = oracle.power_spectrum(x)
+    assert abs(p.sum() - np.mean(np.sum(x * x, axis=1))) < 1e-10            # orthonormal transform: energy is kept
+    c = np.full((N, 2), 1.5)
+    pc = oracle.power_spectrum(c)
+    assert abs(pc[0] - N * 1.5 ** 2) < 1e-10 and np.max(np.abs(pc[1:])) < 1e-20   # a constant has its DC term only
+    n = np.arange(N)
+    k = 7
+    pk = oracle.power_spectrum(np.cos(np.pi * k * (2 * n + 1) / (2 * N))[:, None] * 2.0)
+    want = np.zeros(N)
+    want[k] = 4.0 * N / 2                                                     # alpha_k^2 (sum cos^2)^2 = (2/N)(N/2)^2
+    assert np.max(np.abs(pk - want)) < 1e-10
+
+
+def test_power_spectrum_of_ar1_follows_the_textbook_spectrum():
+    """Many AR(1) channels: the averaged DCT power at component t approaches the AR(1) spectral
+    density (1 - rho^2) / (1 - 2 rho cos w + rho^2) at w = pi t / N (away from the edges)."""
+    N, rho = 256, 0.9
+    e = rng(22).standard_normal((40, N + 200, 16))
+    x = np.zeros_like(e)
+    for i in range(1, N + 200):
+        x[:, i] = rho * x[:, i - 1] + math.sqrt(1 - rho * rho) * e[:, i]
+    p = oracle.power_spectrum(x[:, 200:])
+    w = np.pi * np.arange(N) / N
+    want = (1 - rho * rho) / (1 - 2 * rho * np.cos(w) + rho * rho)
+    band = slice(8, N - 8)
+    assert np.max(np.abs(p[band] / want[band] - 1)) < 0.25                    # 640 channels: ~6 % noise per component
+    assert abs(np.mean(p[band] / want[band]) - 1) < 0.03

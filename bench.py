@@ -355,6 +355,45 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 
+def run_spectrum(args, ctx, fk, synth, dev, peaks):
+    """Average DCT power spectrum of a 7B-shaped cache (Section 3.1): one freqkv_power_spectrum call per step."""
+    w = synth.WORKLOADS["llama2_7b"]
+    cache_len, sink = w.capacity, w.sink
+    n_in = cache_len - sink
+    k, v = synth.make_cache(w, dev)
+    for _ in range(max(args.warmup, 3)):
+        ctx.power_spectrum(k, v, cache_len, sink)
+    torch.cuda.synchronize()
+    ctx.get_timing()
+    ctx.set_timing(True)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        ctx.power_spectrum(k, v, cache_len, sink)
+    b.record()
+    torch.cuda.synchronize()
+    n, t_ms, _ = ctx.get_timing()
+    ctx.set_timing(False)
+    ms = a.elapsed_time(b) / args.steps
+    kernel_ms = t_ms / max(n, 1)
+    nh = (n_in + 1) // 2
+    flops = 2.0 * 2 * nh * nh * w.head_dim * w.n_matrices      # even rows on u, odd rows on v
+    cache_in = w.n_matrices * cache_len * w.head_dim * 2
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    return {"metric": "power-spectrum GB/s of cache in", "value": cache_in / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "spectrum_7b", "batch": w.batch, "layers": w.layers, "kv_heads": w.kv_heads,
+                       "head_dim": w.head_dim, "cache_len": cache_len, "sink": sink,
+                       "step": "one freqkv_power_spectrum call (fold + all N DCT components + squared sums)",
+                       "l2": "inputs larger than L2 (%.2f GB of cache per step)" % (cache_in / 1e9)},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": "sustained, of " + peaks["source"],
+                         "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "kernel": "freqkv_gemm_kernel<spectrum>",
+                         "kernel_ms": kernel_ms, "flops_per_launch": flops, "traffic": None},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -380,6 +419,15 @@ def main():
     from paper_2505_00570_b200 import binding as fk
     from paper_2505_00570_b200 import synth
 
+    if args.workload == "spectrum_7b":
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            ctx = fk.Context(local_rank)
+            print(json.dumps(run_spectrum(args, ctx, fk, synth, torch.device("cuda", local_rank), load_peaks())), flush=True)
+            ctx.close()
+        return
     if args.workload in ("attend_7b", "attend_8b"):   # side workload: the step after the compression path
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")

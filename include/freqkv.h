@@ -117,6 +117,19 @@ freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void
 freqkv_status freqkv_compress_band(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
                                    int32_t kept_len, int32_t sink, int32_t first_component, void* cuda_stream);
 
+/* Average power spectrum of the cached states along the token axis (Section 3.1, the analysis
+ * behind the paper's power-spectrum figures): every channel of rows [sink, cache_len) of every
+ * matrix is transformed with the orthonormal N-point DCT-II of Appendix A (N = cache_len - sink)
+ * and the squared components are averaged over the batch and over head_dim.
+ *   spectrum_k, spectrum_v  DEVICE pointers to fp32 arrays [layers, kv_heads, N], overwritten;
+ *                           either may be NULL (not both).
+ * The cache is only read.  bf16 caches with head_dim 128 (the tensor-core path; components are
+ * computed with bf16 operands and fp32 accumulation); anything else: UNSUPPORTED.  The DCT
+ * matrix of a new N is built on first use and kept by the context (N^2 bytes). */
+freqkv_status freqkv_power_spectrum(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v,
+                                    int32_t cache_len, int32_t sink, float* spectrum_k, float* spectrum_v,
+                                    void* cuda_stream);
+
 /* Ragged form: sequence b holds lens[b] rows and is compressed to sink + kept_len[b] rows,
  * each sequence with the transform of its own length (same definition as above with
  * N = lens[b] - sink, L = kept_len[b]).  `lens` and `kept_len` are host arrays of

@@ -27,7 +27,7 @@ EXPORTS = [
     "freqkv_append", "freqkv_last_device_status", "freqkv_check_compress", "freqkv_check_append",
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
     "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc", "freqkv_attend_decode",
-    "freqkv_check_attend", "freqkv_compress_band",
+    "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.freqkv_plan.argtypes = [c_void_p, c_int32, c_int32, c_int, c_int, c_void_p]
         L.freqkv_compress.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
         L.freqkv_compress_band.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p]
+        L.freqkv_power_spectrum.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.freqkv_compress_ragged.argtypes = [c_void_p, LP, c_void_p, c_void_p, I32P, I32P, c_int32, c_void_p]
         L.freqkv_append.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P, c_void_p]
         L.freqkv_last_device_status.argtypes = [c_void_p, c_void_p]
@@ -220,6 +221,20 @@ class Context:
                                         first_component, _stream_ptr(stream))
         self._check(st, "freqkv_compress_band")
         return sink + kept_len
+
+    def power_spectrum(self, k: torch.Tensor, v: torch.Tensor, cache_len: int, sink: int, stream=None):
+        """Average DCT power spectrum of rows [sink, cache_len) over batch and channels:
+        (spectrum_k, spectrum_v), each fp32 ``[layers, kv_heads, cache_len - sink]`` on the cache's device."""
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        n = max(cache_len - sink, 0)
+        sk = torch.empty(lay.layers, lay.kv_heads, n, dtype=torch.float32, device=k.device)
+        sv = torch.empty_like(sk)
+        st = lib().freqkv_power_spectrum(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), cache_len, sink,
+                                         sk.data_ptr(), sv.data_ptr(), _stream_ptr(stream))
+        self._check(st, "freqkv_power_spectrum")
+        return sk, sv
 
     def compress_ragged(self, k: torch.Tensor, v: torch.Tensor, lens: list[int], kept_len: list[int], sink: int,
                         stream=None) -> list[int]:

@@ -53,6 +53,7 @@ struct freqkv_ctx {
 namespace {
 
 constexpr size_t kScratchChunkBytes = size_t(1) << 30;  // per-chunk output staging of the scratch paths
+constexpr int32_t kDctRows = -1;  // plan key of the plain DCT matrix (power spectrum) among the retained-band offsets
 constexpr size_t kBasisBudgetBytes = size_t(12) << 30;  // plan cache is flushed beyond this
 
 struct DeviceGuard {
@@ -232,7 +233,8 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
             ctx->kernels_launched += 1;
         }
         if (e == cudaSuccess && pb) {
-            e = launch_build_folded_basis(pb, n_in, n_keep, first, b.fold_ld, b.fold_rows_pad, stream);
+            e = first == kDctRows ? launch_build_dct_folded(pb, n_in, b.fold_ld, b.fold_rows_pad, stream)
+                                  : launch_build_folded_basis(pb, n_in, n_keep, first, b.fold_ld, b.fold_rows_pad, stream);
             ctx->kernels_launched += 1;
         }
         if (e != cudaSuccess) {
@@ -564,6 +566,42 @@ freqkv_status freqkv_compress_band(freqkv_ctx* ctx, const freqkv_layout* layout,
     if (!g.ok) return FREQKV_ERR_CUDA;
     return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
                           static_cast<cudaStream_t>(cuda_stream), first_component);
+}
+
+freqkv_status freqkv_power_spectrum(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v,
+                                    int32_t cache_len, int32_t sink, float* spectrum_k, float* spectrum_v, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = freqkv_check_compress(layout, k, v, cache_len, 0, sink);
+    if (st != FREQKV_OK) return st;
+    if (!spectrum_k && !spectrum_v) return FREQKV_ERR_INVALID_ARG;
+    const freqkv_layout& l = *layout;
+    const int32_t n_in = cache_len - sink;
+    if (n_in < 1) return FREQKV_ERR_INVALID_ARG;
+    if (!gemm_supported(l.dtype, l.head_dim, n_in, n_in)) return FREQKV_ERR_UNSUPPORTED;  // bf16, head_dim 128
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    Basis basis;
+    st = get_basis(ctx, n_in, n_in, kDctRows, false, true, stream, &basis);
+    if (st != FREQKV_OK) return st;
+    const size_t bytes = (size_t)l.layers * l.kv_heads * n_in * sizeof(float);
+    if (spectrum_k) FREQKV_CUDA(ctx, cudaMemsetAsync(spectrum_k, 0, bytes, stream));
+    if (spectrum_v) FREQKV_CUDA(ctx, cudaMemsetAsync(spectrum_v, 0, bytes, stream));
+    SpectrumOut out;
+    out.k = spectrum_k;
+    out.v = spectrum_v;
+    out.scale = 1.0f / ((float)l.batch * (float)l.head_dim);
+    const CacheView view = make_view(l, const_cast<void*>(k), const_cast<void*>(v), 0, l.batch);
+    TransformTimer timer(ctx, stream, false);
+    LaunchHooks hooks;
+    hooks.user = &timer;
+    hooks.before = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->begin(); };
+    hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
+    const cudaError_t e = launch_gemm(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream, &out);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
+    ctx->kernels_launched += ctx->gemm.kernels_last_call;
+    return FREQKV_OK;
 }
 
 freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t* lens,

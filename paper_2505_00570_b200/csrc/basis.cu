@@ -13,6 +13,8 @@
 // 0 < a+ < 4LN and |a-| < 2LN, so the denominator vanishes only at a- = 0.  The numerator's
 // phase is reduced exactly in 64-bit integers modulo 8LN before sinpi, so every entry is
 // accurate to a few fp64 ulps; it is rounded once to fp32 and once to bf16.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace freqkv {
@@ -105,7 +107,35 @@ __global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32
     }
 }
 
+// The plain orthonormal DCT-II of length N, folded the same way (power-spectrum analysis): plane 0
+// holds the even rows C[2m][n], plane 1 the odd rows C[2m+1][n], n < ceil(N/2); applied to
+// u_n = x_n + x_{N-1-n} and v_n = x_n - x_{N-1-n} they give the components z_2m and z_2m+1 (for odd N the
+// middle column meets u = x once; the odd rows vanish there).  C[t][n] = alpha_t cos(pi t (2n+1) / (2N)),
+// the phase t (2n+1) reduced exactly modulo 4N.
+__global__ void build_dct_folded_kernel(__nv_bfloat16* __restrict__ out, int32_t n_in, int32_t ld, int32_t rows_pad)
+{
+    const int64_t plane = (int64_t)rows_pad * ld;
+    const int64_t N = n_in, Nh = (N + 1) / 2;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < 2 * plane; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t eo = i / plane, j = i % plane, m = j / ld, n = j % ld, t = 2 * m + eo;
+        double c = 0.0;
+        if (t < N && n < Nh) {
+            const int64_t k = (t * (2 * n + 1)) % (4 * N);
+            c = (t == 0 ? sqrt(1.0 / (double)N) : sqrt(2.0 / (double)N)) * cospi((double)k / (double)(2 * N));
+        }
+        out[i] = __double2bfloat16(c);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_build_dct_folded(__nv_bfloat16* out, int32_t n_in, int32_t ld, int32_t rows_pad, cudaStream_t stream)
+{
+    const int64_t total = (int64_t)2 * rows_pad * ld;
+    int64_t blocks = std::min<int64_t>((total + 255) / 256, 148 * 32);
+    build_dct_folded_kernel<<<(unsigned)std::max<int64_t>(blocks, 1), 256, 0, stream>>>(out, n_in, ld, rows_pad);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t first, int32_t ld,
                                       int32_t rows_pad, cudaStream_t stream)

@@ -56,6 +56,9 @@ cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in
 cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t first, int32_t ld,
                                       int32_t rows_pad, cudaStream_t stream);
 
+// Even rows | odd rows of the orthonormal N-point DCT-II, restricted to n < ceil(N/2) (two planes of rows_pad x ld).
+cudaError_t launch_build_dct_folded(__nv_bfloat16* out, int32_t n_in, int32_t ld, int32_t rows_pad, cudaStream_t stream);
+
 // scratch[i - first][m][c] = sum_n P[m][n] * X_i[sink + n][c] for matrices first .. first+count-1.
 cudaError_t launch_project_simt(const CacheView& view, int32_t dtype, int32_t first, int32_t count, const Basis& basis,
                                 int32_t sink, void* scratch, cudaStream_t stream);

@@ -72,6 +72,10 @@ struct GemmParams {
     int32_t m_pairs, k_steps;   // tiles of 256 folded rows per (batch, layer, kv_head); slices per phase
     int32_t sink;
     int32_t mirror_sign;        // +1: y[L-1-m] = s - d;  -1: y[L-1-m] = d - s (a retained band that starts at an odd component)
+    // power-spectrum mode only: per tensor [layers][kv_heads][n_in] sums, the weight of one squared value
+    float* spectrum[2];
+    float spectrum_scale;
+    int32_t n_in;
     int32_t* status;
 };
 
@@ -315,6 +319,11 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
     }
 }
 
+// SPECTRUM = false: the compression above.  SPECTRUM = true: the basis holds the even and the odd
+// rows of the plain N-point DCT-II instead of Pe and Po, so S and D are the components z_2m and
+// z_2m+1 themselves; the epilogue squares them, sums over the 128 channels of its tensor and adds
+// the sum to the power spectrum of its (layer, kv head).  Nothing is written to the cache.
+template <bool SPECTRUM>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_x,
                    const CacheView view, const GemmParams prm)
@@ -436,6 +445,38 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tensor * 128;
         const uint32_t leader_s_empty = cluster_addr(acc_empty_bar(0), 0), leader_d_empty = cluster_addr(acc_empty_bar(1), 0);
         uint32_t tile_no = 0;
+        if constexpr (SPECTRUM) {
+            for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
+                const int32_t pair = prm.pair0 + tile / prm.m_pairs;
+                const int32_t head = pair % view.kv_heads, layer = (pair / view.kv_heads) % view.layers;
+                const int32_t m = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
+                bool alive = true;
+                for (int eo = 0; eo < 2; ++eo) {
+                    if (!mbar_wait(acc_full_bar(eo), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) {
+                        alive = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    float sum = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32<0>(lane_addr + eo * 256 + c * 32, r);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), sum);
+                    }
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(eo ? leader_d_empty : leader_s_empty);
+                    const int32_t t = 2 * m + eo;  // S holds the even components, D the odd ones
+                    if (t < prm.n_in && prm.spectrum[tensor])
+                        atomicAdd(prm.spectrum[tensor] + ((int64_t)layer * view.kv_heads + head) * prm.n_in + t,
+                                  sum * prm.spectrum_scale);
+                }
+                if (!alive) break;
+            }
+        } else
         for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
             // S = Pe U: park this thread's row (128 columns) in registers, release that half
             if (!mbar_wait(acc_full_bar(0), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
@@ -555,7 +596,7 @@ bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_kee
 }
 
 cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
-                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream)
+                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream, const SpectrumOut* spectrum)
 {
     state->kernels_last_call = 0;
     state->last_error = nullptr;
@@ -564,7 +605,9 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         return cudaErrorNotSupported;
     }
     if (!state->attr_set) {
-        const cudaError_t e = cudaFuncSetAttribute(freqkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(freqkv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(freqkv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) {
             state->last_error = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -582,7 +625,7 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        const cudaError_t q = cudaOccupancyMaxActiveClusters(&n, freqkv_gemm_kernel, &cfg);
+        const cudaError_t q = cudaOccupancyMaxActiveClusters(&n, freqkv_gemm_kernel<false>, &cfg);
         if (q != cudaSuccess || n < 1) {
             state->last_error = "cudaOccupancyMaxActiveClusters: no CTA pair fits on this device";
             return q != cudaSuccess ? q : cudaErrorLaunchOutOfResources;
@@ -649,6 +692,10 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         prm.k_steps = (n_half + BK - 1) / BK;
         prm.sink = sink;
         prm.mirror_sign = (basis.first & 1) ? -1 : 1;
+        prm.spectrum[0] = spectrum ? spectrum->k : nullptr;
+        prm.spectrum[1] = spectrum ? spectrum->v : nullptr;
+        prm.spectrum_scale = spectrum ? spectrum->scale : 0.f;
+        prm.n_in = basis.n_in;
         prm.status = status_dev;
         const int32_t tiles = job.pair_count * m_pairs;
         const int clusters = std::min<int32_t>(tiles, state->max_clusters);
@@ -665,7 +712,8 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (hooks.before) hooks.before(hooks.user, stream);
-        e = cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel, map_p, map_x, view, prm);
+        e = spectrum ? cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<true>, map_p, map_x, view, prm)
+                     : cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<false>, map_p, map_x, view, prm);
         if (hooks.after) hooks.after(hooks.user, stream);
         if (e != cudaSuccess) {
             state->last_error = "freqkv_gemm_kernel launch";

@@ -21,9 +21,17 @@ struct LaunchHooks {
     void* user = nullptr;
 };
 
+// Power-spectrum mode: device arrays [layers][kv_heads][n_in] (either may be null) that receive
+// scale * (sum over the 128 channels of the squared DCT components), accumulated over the batch.
+struct SpectrumOut {
+    float* k = nullptr;
+    float* v = nullptr;
+    float scale = 1.f;
+};
+
 bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_keep);
 cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
-                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
+                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream, const SpectrumOut* spectrum = nullptr);
 void gemm_release(GemmState* state);
 
 }  // namespace freqkv

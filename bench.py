@@ -261,6 +261,52 @@ def run_ragged(args, ctx, fk, synth, w, dev, peaks):
             "cpu_baseline": None, "e2e": None, "gpu_launches": None}
 
 
+def run_stream_graph(args, ctx, fk, synth, w, dev, peaks, total_tokens=32768):
+    """Config 4 through the decode graph: lengths on the device, the trigger and the compression
+    inside the graph; per step the host only refills the staging rows and launches the graph."""
+    cap, sink = w.capacity, w.sink
+    kept = w.kept_len(cap)
+    k, v = synth.make_cache(w, dev, fill_len=0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed)
+    scales = synth.channel_scales(w, gen, dev)
+    ring, _ = synth.ar1_rows(w, 64, gen, dev, scales)
+    toks = [ring[:, :, :, j:j + 1].contiguous() for j in range(64)]
+    lens = torch.zeros(w.batch, dtype=torch.int32, device=dev)
+    stage_k, stage_v = torch.empty_like(toks[0]), torch.empty_like(toks[0])
+    graph = fk.DecodeGraph(ctx, k, v, stage_k, stage_v, lens, kept, sink)
+    for t in range(8):   # warm-up launches on a scratch run, then reset
+        stage_k.copy_(toks[t]); stage_v.copy_(toks[t]); graph.launch()
+    lens.zero_()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    a.record()
+    for t in range(total_tokens):
+        nk = toks[t & 63]
+        stage_k.copy_(nk)
+        stage_v.copy_(nk)
+        graph.launch()
+    b.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    final = lens.tolist()
+    graph.close()
+    count = 0 if total_tokens <= cap else 1 + (total_tokens - cap - 1) // (cap - sink - kept)  # fills after the first one
+    per_tok_us = wall / total_tokens * 1e6
+    e = 2
+    cache_in = w.n_matrices * cap * w.head_dim * e
+    return {"metric": METRIC, "value": cache_in * count / wall / 1e9, "unit": UNIT, "n_gpus": 1, "steps": total_tokens,
+            "warmup": 8, "ms_per_step": wall / total_tokens * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name + "_graph", "batch": w.batch, "layers": w.layers, "kv_heads": w.kv_heads,
+                       "head_dim": w.head_dim, "capacity": cap, "sink": sink, "kept_len": kept, "tokens": total_tokens,
+                       "step": "staging rows refilled + one freqkv_decode_graph_launch (device-side trigger)"},
+            "stream": {"compressions": count, "final_lens": final[:2], "wall_s": wall, "device_ms": a.elapsed_time(b),
+                       "amortised_us_per_token_step": per_tok_us, "amortised_us_per_token_per_sequence": per_tok_us / w.batch},
+            "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": None}
+
+
 def run_stream(args, ctx, fk, synth, w, dev, peaks, total_tokens=32768):
     """Config 4: tokens appended one per step from empty caches; a full cache is compressed to
     half its non-sink length before the next token goes in.  Reports the amortised time per
@@ -447,7 +493,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     n_gpus = world
 
-    w = synth.WORKLOADS[args.workload]
+    w = synth.WORKLOADS["stream_7b" if args.workload == "stream_7b_graph" else args.workload]
     if args.layers > 0:
         import dataclasses
 
@@ -461,9 +507,9 @@ def main():
     ctx = fk.Context(local_rank)
     variant = {"auto": fk.AUTO, "gemm": fk.GEMM, "fdct": fk.FDCT, "simt": fk.SIMT}[args.variant]
     ctx.set_variant(variant)
-    if args.workload in ("ragged_8b", "stream_7b"):   # side workloads: one line each, single GPU
+    if args.workload in ("ragged_8b", "stream_7b", "stream_7b_graph"):   # side workloads: one line each, single GPU
         if rank == 0:
-            fn = run_ragged if args.workload == "ragged_8b" else run_stream
+            fn = {"ragged_8b": run_ragged, "stream_7b": run_stream, "stream_7b_graph": run_stream_graph}[args.workload]
             print(json.dumps(fn(args, ctx, fk, synth, w, dev, load_peaks())), flush=True)
         ctx.close()
         return

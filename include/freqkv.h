@@ -148,6 +148,28 @@ freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layou
 freqkv_status freqkv_append(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
                             const void* new_v, int32_t n_new, int32_t* lens, void* cuda_stream);
 
+/* One decode step as a replayable CUDA graph, with the cache lengths on the DEVICE: no host
+ * round trip decides when to compress (Section 3.4: the incoming token is appended; when the
+ * cache is full it is compressed first).  For uniform batches: every sequence has the same length.
+ *   lens_device   DEVICE array of `batch` int32 lengths, read and updated by the graph;
+ *   new_k, new_v  DEVICE staging rows, dense [batch, layers, kv_heads, 1, head_dim]; the caller
+ *                 refills them (on the launching stream) before each launch.
+ * Each launch runs: a one-thread trigger kernel; if every sequence holds `capacity` rows, the
+ * compression of rows [sink, capacity) to kept_len rows (tensor-core variant) and lens := sink +
+ * kept_len -- skipped otherwise by a conditional graph node; then the append of the staged row at
+ * lens[b] and lens[b] += 1.  If some but not all sequences are full, nothing is compressed, the
+ * full ones are skipped and freqkv_last_device_status reports FREQKV_ERR_CAPACITY.
+ * create allocates and builds everything the step needs (plan, scratch, graph) and may
+ * synchronise the device; launch only enqueues the graph on `cuda_stream`.  The pointers are
+ * baked into the graph.  Requirements: bf16, head_dim 128, 1 <= kept_len < capacity - sink.
+ * destroy synchronises the device.  A graph must be destroyed before its context. */
+typedef struct freqkv_decode_graph freqkv_decode_graph;
+freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
+                                         const void* new_v, int32_t* lens_device, int32_t kept_len, int32_t sink,
+                                         freqkv_decode_graph** out);
+freqkv_status freqkv_decode_graph_launch(freqkv_decode_graph* graph, void* cuda_stream);
+freqkv_status freqkv_decode_graph_destroy(freqkv_decode_graph* graph);
+
 /* Host-buffer form of freqkv_compress for callers whose cache lives in host memory (pinned
  * memory gives full copy bandwidth; pageable memory works).  k_host / v_host use `layout` in
  * host memory.  Rows [sink, cache_len) of every matrix are copied to a device staging cache the

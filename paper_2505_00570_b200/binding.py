@@ -28,6 +28,7 @@ EXPORTS = [
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
     "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc", "freqkv_attend_decode",
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
+    "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -71,6 +72,10 @@ def lib() -> ctypes.CDLL:
         L.freqkv_compress.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
         L.freqkv_compress_band.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p]
         L.freqkv_power_spectrum.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
+        L.freqkv_decode_graph_create.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int32,
+                                                 c_int32, POINTER(c_void_p)]
+        L.freqkv_decode_graph_launch.argtypes = [c_void_p, c_void_p]
+        L.freqkv_decode_graph_destroy.argtypes = [c_void_p]
         L.freqkv_compress_ragged.argtypes = [c_void_p, LP, c_void_p, c_void_p, I32P, I32P, c_int32, c_void_p]
         L.freqkv_append.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, I32P, c_void_p]
         L.freqkv_last_device_status.argtypes = [c_void_p, c_void_p]
@@ -154,6 +159,45 @@ def compress_noalloc(k: torch.Tensor, v: torch.Tensor, cache_len: int, kept_len:
     if st != OK:
         raise FreqKVError(st, f"freqkv_compress_noalloc: {status_string(st)}")
     return sink + kept_len
+
+
+class DecodeGraph:
+    """``freqkv_decode_graph``: one decode step (device-side trigger, compression when the cache is
+    full, append of the staged row) replayed as a CUDA graph.  ``lens`` is an int32 device tensor
+    the graph updates; ``new_k`` / ``new_v`` are the staging rows the caller refills before ``launch``."""
+
+    def __init__(self, ctx: "Context", k: torch.Tensor, v: torch.Tensor, new_k: torch.Tensor, new_v: torch.Tensor,
+                 lens: torch.Tensor, kept_len: int, sink: int):
+        lay = layout_of(k)
+        if lens.dtype != torch.int32 or not lens.is_cuda or lens.numel() != lay.batch or not lens.is_contiguous():
+            raise FreqKVError(ERR_INVALID_ARG, "lens must be a dense int32 device tensor with one entry per sequence")
+        want = (k.shape[0], k.shape[1], k.shape[2], 1, k.shape[4])
+        if tuple(new_k.shape) != want or tuple(new_v.shape) != want or not (new_k.is_contiguous() and new_v.is_contiguous()) \
+                or new_k.dtype != k.dtype or new_v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "staging rows must be dense [batch, layers, kv_heads, 1, head_dim] in the cache dtype")
+        self._keep = (ctx, k, v, new_k, new_v, lens)   # the graph holds raw pointers into these
+        self._h = c_void_p()
+        st = lib().freqkv_decode_graph_create(ctx._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), new_k.data_ptr(),
+                                              new_v.data_ptr(), lens.data_ptr(), kept_len, sink, ctypes.byref(self._h))
+        if st != OK:
+            self._h = c_void_p()
+            ctx._check(st, "freqkv_decode_graph_create")
+
+    def launch(self, stream=None):
+        st = lib().freqkv_decode_graph_launch(self._h, _stream_ptr(stream))
+        if st != OK:
+            raise FreqKVError(st, f"freqkv_decode_graph_launch: {status_string(st)}")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().freqkv_decode_graph_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Context:

@@ -831,6 +831,120 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
     return FREQKV_OK;
 }
 
+struct freqkv_decode_graph {
+    freqkv_ctx* ctx = nullptr;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+};
+
+freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
+                                         const void* new_v, int32_t* lens_device, int32_t kept_len, int32_t sink,
+                                         freqkv_decode_graph** out)
+{
+    if (!ctx || !out || !lens_device) return FREQKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    const freqkv_layout& l = *layout;
+    st = check_tensors(l, k, v);
+    if (st != FREQKV_OK) return st;
+    if (!new_k || !new_v) return FREQKV_ERR_INVALID_ARG;
+    if (((uintptr_t)new_k | (uintptr_t)new_v | (uintptr_t)lens_device) & 15) return FREQKV_ERR_UNSUPPORTED;
+    st = check_lengths(l, l.capacity, kept_len, sink);
+    if (st != FREQKV_OK) return st;
+    const int32_t n_in = l.capacity - sink;
+    if (kept_len < 1 || kept_len >= n_in) return FREQKV_ERR_INVALID_ARG;  // a compression must make room
+    if (!gemm_applicable(l, n_in, kept_len)) return FREQKV_ERR_UNSUPPORTED;  // the graph holds the tensor-core variant
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+
+    // everything that allocates or builds tables happens here, outside the graph
+    cudaStream_t cs = nullptr;
+    FREQKV_CUDA(ctx, cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
+    Basis basis;
+    st = get_basis(ctx, n_in, kept_len, 0, false, true, cs, &basis);
+    cudaError_t e = st == FREQKV_OK ? cudaStreamSynchronize(cs) : cudaSuccess;
+    if (st == FREQKV_OK && e == cudaSuccess) e = gemm_prepare(&ctx->gemm, l.batch * l.layers * l.kv_heads, basis, ctx->sm_count);
+    freqkv_decode_graph* dg = new (std::nothrow) freqkv_decode_graph();
+    auto fail = [&](freqkv_status code, cudaError_t ce, const char* where) {
+        if (ce != cudaSuccess) code = cuda_fail(ctx, ce, where);
+        if (dg) {
+            if (dg->exec) cudaGraphExecDestroy(dg->exec);
+            if (dg->graph) cudaGraphDestroy(dg->graph);
+            delete dg;
+        }
+        cudaStreamDestroy(cs);
+        cudaGetLastError();
+        return code;
+    };
+    if (st != FREQKV_OK) return fail(st, cudaSuccess, "");
+    if (e != cudaSuccess) return fail(FREQKV_ERR_CUDA, e, "decode graph set-up");
+    if (!dg) return fail(FREQKV_ERR_ALLOC, cudaSuccess, "");
+    dg->ctx = ctx;
+
+    // graph: trigger -> IF (all sequences full) { fold, GEMM, lengths := sink + kept_len } -> append + advance
+    if ((e = cudaGraphCreate(&dg->graph, 0)) != cudaSuccess) return fail(FREQKV_ERR_CUDA, e, "cudaGraphCreate");
+    cudaGraphConditionalHandle handle;
+    if ((e = cudaGraphConditionalHandleCreate(&handle, dg->graph, 0, cudaGraphCondAssignDefault)) != cudaSuccess)
+        return fail(FREQKV_ERR_CUDA, e, "cudaGraphConditionalHandleCreate");
+    cudaGraphNode_t trigger = nullptr, branch = nullptr;
+    if ((e = add_decode_trigger_node(dg->graph, &trigger, lens_device, l.batch, l.capacity, handle, ctx->status_dev)) != cudaSuccess)
+        return fail(FREQKV_ERR_CUDA, e, "trigger node");
+    cudaGraphNodeParams cond = {};
+    cond.type = cudaGraphNodeTypeConditional;
+    cond.conditional.handle = handle;
+    cond.conditional.type = cudaGraphCondTypeIf;
+    cond.conditional.size = 1;
+    if ((e = cudaGraphAddNode(&branch, dg->graph, &trigger, 1, &cond)) != cudaSuccess)
+        return fail(FREQKV_ERR_CUDA, e, "conditional node");
+    cudaGraph_t body = cond.conditional.phGraph_out[0];
+    const bool was_timing = ctx->timing;
+    ctx->timing = false;  // event records do not belong in the graph
+    if ((e = cudaStreamBeginCaptureToGraph(cs, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed)) != cudaSuccess) {
+        ctx->timing = was_timing;
+        return fail(FREQKV_ERR_CUDA, e, "capture of the compression");
+    }
+    st = compress_group(ctx, l, k, v, 0, l.batch, n_in, kept_len, sink, FREQKV_GEMM, cs);
+    e = st == FREQKV_OK ? launch_decode_set_lens(lens_device, l.batch, sink + kept_len, cs) : cudaSuccess;
+    cudaGraph_t captured = nullptr;
+    const cudaError_t e_end = cudaStreamEndCapture(cs, &captured);
+    ctx->timing = was_timing;
+    if (st != FREQKV_OK) return fail(st, cudaSuccess, "");
+    if (e != cudaSuccess || e_end != cudaSuccess) return fail(FREQKV_ERR_CUDA, e != cudaSuccess ? e : e_end, "capture of the compression");
+    // the append, after the branch
+    if ((e = cudaStreamBeginCaptureToGraph(cs, dg->graph, &branch, nullptr, 1, cudaStreamCaptureModeRelaxed)) != cudaSuccess)
+        return fail(FREQKV_ERR_CUDA, e, "capture of the append");
+    e = launch_decode_append(make_view(l, k, v, 0, l.batch), l.dtype, l.batch, lens_device, l.capacity, new_k, new_v, cs);
+    const cudaError_t e_end2 = cudaStreamEndCapture(cs, &captured);
+    if (e != cudaSuccess || e_end2 != cudaSuccess) return fail(FREQKV_ERR_CUDA, e != cudaSuccess ? e : e_end2, "capture of the append");
+    if ((e = cudaGraphInstantiate(&dg->exec, dg->graph, 0)) != cudaSuccess) return fail(FREQKV_ERR_CUDA, e, "cudaGraphInstantiate");
+    cudaStreamDestroy(cs);
+    *out = dg;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_decode_graph_launch(freqkv_decode_graph* graph, void* cuda_stream)
+{
+    if (!graph || !graph->exec) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(graph->ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    FREQKV_CUDA(graph->ctx, cudaGraphLaunch(graph->exec, static_cast<cudaStream_t>(cuda_stream)));
+    graph->ctx->kernels_launched += 3;  // trigger, append, advance (the compression adds 3 when it runs)
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_decode_graph_destroy(freqkv_decode_graph* graph)
+{
+    if (!graph) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(graph->ctx->device);
+    cudaDeviceSynchronize();
+    if (graph->exec) cudaGraphExecDestroy(graph->exec);
+    if (graph->graph) cudaGraphDestroy(graph->graph);
+    cudaGetLastError();
+    delete graph;
+    return FREQKV_OK;
+}
+
 freqkv_status freqkv_set_timing(freqkv_ctx* ctx, int32_t enabled)
 {
     if (!ctx) return FREQKV_ERR_INVALID_ARG;
@@ -872,7 +986,12 @@ freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream)
     FREQKV_CUDA(ctx, cudaMemsetAsync(ctx->status_dev, 0, sizeof(word), stream));
     FREQKV_CUDA(ctx, cudaStreamSynchronize(stream));
     if (word != 0) {
-        char buf[96];
+        char buf[128];
+        if (word == DECODE_ERR_MIXED_LENGTHS) {
+            snprintf(buf, sizeof(buf), "decode graph: some but not all sequences were full; the full ones were not appended to");
+            ctx->last_error = buf;
+            return FREQKV_ERR_CAPACITY;
+        }
         snprintf(buf, sizeof(buf), "device status word 0x%08x (a bounded wait gave up)", (unsigned)word);
         ctx->last_error = buf;
         return FREQKV_ERR_TIMEOUT;

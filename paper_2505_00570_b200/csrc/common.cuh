@@ -71,6 +71,15 @@ cudaError_t launch_copy_back(const CacheView& view, int32_t dtype, int32_t first
 cudaError_t launch_append(const CacheView& view, int32_t dtype, int32_t batch, const int32_t* lens_host,
                           int32_t n_new, const void* new_k, const void* new_v, cudaStream_t stream);
 
+// Decode step with device-resident lengths (pieces of the graph api.cu builds).
+constexpr int32_t DECODE_ERR_MIXED_LENGTHS = 0x100;  // status-word bit: some but not all sequences were full
+cudaError_t add_decode_trigger_node(cudaGraph_t graph, cudaGraphNode_t* node, const int32_t* lens, int32_t batch,
+                                    int32_t capacity, cudaGraphConditionalHandle handle, int32_t* status);
+cudaError_t launch_decode_set_lens(int32_t* lens, int32_t batch, int32_t value, cudaStream_t stream);
+// rows at lens[b] <- the new rows ([batch, layers, kv_heads, 1, head_dim]), then lens[b] += 1 (full sequences skipped)
+cudaError_t launch_decode_append(const CacheView& view, int32_t dtype, int32_t batch, int32_t* lens, int32_t capacity,
+                                 const void* new_k, const void* new_v, cudaStream_t stream);
+
 inline size_t dtype_size(int32_t dtype) { return dtype == FREQKV_F32 ? 4 : 2; }
 
 }  // namespace freqkv

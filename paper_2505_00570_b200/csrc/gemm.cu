@@ -595,10 +595,11 @@ bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_kee
     return dtype == FREQKV_BF16 && head_dim == 128 && n_in >= 1 && n_keep >= 1 && n_keep <= n_in;
 }
 
-cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
-                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream, const SpectrumOut* spectrum)
+// Everything a launch needs that is not a stream operation: kernel attributes, the count of
+// resident CTA pairs, the scratch buffer for `pairs` (batch, layer, kv_head) triples of this basis.
+// launch_gemm calls it itself; a caller that must not allocate later (stream capture) calls it first.
+cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, int sm_count)
 {
-    state->kernels_last_call = 0;
     state->last_error = nullptr;
     if (!encode_fn()) {
         state->last_error = "cuTensorMapEncodeTiled is not available from this driver";
@@ -633,15 +634,10 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         state->max_clusters = std::min(n, sm_count / 2);
         state->attr_set = true;
     }
-    const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
-    const int32_t m_pairs = (rows_half + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
-    const int32_t pairs = view.mats_per_tensor;
+    const int32_t n_half = (basis.n_in + 1) / 2;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;  // K and V, U and V planes
-
-    // One pass when the folded inputs fit the scratch buffer, else several passes of `chunk` pairs.
     const int64_t fit = std::max<int64_t>(1, (int64_t)(kFoldBufferBytes / per_pair));
-    const int64_t chunk = std::min<int64_t>(fit, pairs);
-    const size_t need = (size_t)chunk * per_pair;
+    const size_t need = (size_t)std::min<int64_t>(fit, pairs) * per_pair;
     if (need > state->scratch_bytes) {
         if (state->scratch) {
             cudaError_t e = cudaDeviceSynchronize();
@@ -657,6 +653,21 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         }
         state->scratch_bytes = need;
     }
+    return cudaSuccess;
+}
+
+cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
+                        int sm_count, const LaunchHooks& hooks, cudaStream_t stream, const SpectrumOut* spectrum)
+{
+    state->kernels_last_call = 0;
+    const cudaError_t prepared = gemm_prepare(state, view.mats_per_tensor, basis, sm_count);
+    if (prepared != cudaSuccess) return prepared;
+    const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
+    const int32_t m_pairs = (rows_half + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
+    const int32_t pairs = view.mats_per_tensor;
+    const size_t per_pair = (size_t)4 * n_half * 128 * 2;
+    // One pass when the folded inputs fit the scratch buffer, else several passes of `chunk` pairs.
+    const int64_t chunk = std::min<int64_t>(std::max<int64_t>(1, (int64_t)(kFoldBufferBytes / per_pair)), pairs);
     CUtensorMap map_p;
     if (!encode_basis_map(&map_p, basis)) {
         state->last_error = "tensor map encoding rejected the basis";

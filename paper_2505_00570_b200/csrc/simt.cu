@@ -183,6 +183,54 @@ __global__ void __launch_bounds__(256) append_rows_kernel(CacheView view, int32_
     }
 }
 
+// ---- decode step with the lengths on the device (replayed as a CUDA graph, see api.cu) ----
+
+// One thread: decide whether this step must compress first.  Every sequence full -> the
+// conditional body (the compression) runs; none full -> it is skipped; some but not all full ->
+// the batch is not uniform, which this path does not take: an error bit is set, nothing is
+// compressed and the full sequences are not appended to.
+__global__ void decode_trigger_kernel(const int32_t* __restrict__ lens, int32_t batch, int32_t capacity,
+                                      cudaGraphConditionalHandle handle, int32_t* status)
+{
+    int32_t full = 0;
+    for (int32_t b = 0; b < batch; ++b) full += lens[b] >= capacity;
+    if (full != 0 && full != batch) atomicOr(status, DECODE_ERR_MIXED_LENGTHS);
+    cudaGraphSetConditional(handle, full == batch ? 1u : 0u);
+}
+
+__global__ void decode_set_lens_kernel(int32_t* lens, int32_t batch, int32_t value)
+{
+    const int32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch) lens[b] = value;
+}
+
+// One new row per matrix, written at the sequence's device-resident length (full sequences are skipped).
+__global__ void decode_append_kernel(CacheView view, int32_t batch, const int32_t* __restrict__ lens, int32_t capacity,
+                                     int32_t elt_size, const uint4* __restrict__ new_k, const uint4* __restrict__ new_v)
+{
+    const int32_t vec_per_row = view.head_dim * elt_size / 16;
+    const int32_t mats = batch * view.layers * view.kv_heads;
+    const int64_t per_tensor = (int64_t)mats * vec_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < 2 * per_tensor;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t tensor = i >= per_tensor;
+        const int64_t j = i - tensor * per_tensor;
+        const int32_t vcol = (int32_t)(j % vec_per_row), idx = (int32_t)(j / vec_per_row);
+        const int32_t b = idx / (view.layers * view.kv_heads);
+        const int32_t len = lens[b];
+        if (len >= capacity) continue;
+        const int64_t off = matrix_offset(view, idx) + (int64_t)len * view.stride_token;
+        char* dst = static_cast<char*>(tensor_base(view, tensor)) + off * elt_size;
+        reinterpret_cast<uint4*>(dst)[vcol] = (tensor ? new_v : new_k)[j];
+    }
+}
+
+__global__ void decode_advance_kernel(int32_t* lens, int32_t batch, int32_t capacity)
+{
+    const int32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch && lens[b] < capacity) lens[b] += 1;
+}
+
 unsigned grid_for(int64_t work_items, int threads)
 {
     int64_t blocks = (work_items + threads - 1) / threads;
@@ -217,6 +265,38 @@ cudaError_t launch_copy_back(const CacheView& view, int32_t dtype, int32_t first
     const int64_t total = (int64_t)count * n_keep * (view.head_dim * elt / 16);
     copy_back_kernel<<<grid_for(total, 256), 256, 0, stream>>>(view, first, count, n_keep, sink, elt,
                                                                static_cast<const uint4*>(scratch));
+    return cudaGetLastError();
+}
+
+cudaError_t add_decode_trigger_node(cudaGraph_t graph, cudaGraphNode_t* node, const int32_t* lens, int32_t batch,
+                                    int32_t capacity, cudaGraphConditionalHandle handle, int32_t* status)
+{
+    void* args[] = {(void*)&lens, (void*)&batch, (void*)&capacity, (void*)&handle, (void*)&status};
+    cudaKernelNodeParams kp = {};
+    kp.func = (void*)decode_trigger_kernel;
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(1);
+    kp.kernelParams = args;
+    return cudaGraphAddKernelNode(node, graph, nullptr, 0, &kp);
+}
+
+cudaError_t launch_decode_set_lens(int32_t* lens, int32_t batch, int32_t value, cudaStream_t stream)
+{
+    decode_set_lens_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(lens, batch, value);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_append(const CacheView& view, int32_t dtype, int32_t batch, int32_t* lens, int32_t capacity,
+                                 const void* new_k, const void* new_v, cudaStream_t stream)
+{
+    const int32_t elt = (int32_t)dtype_size(dtype);
+    const int64_t vecs = (int64_t)2 * batch * view.layers * view.kv_heads * (view.head_dim * elt / 16);
+    decode_append_kernel<<<grid_for(vecs, 256), 256, 0, stream>>>(view, batch, lens, capacity, elt,
+                                                                  static_cast<const uint4*>(new_k),
+                                                                  static_cast<const uint4*>(new_v));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    decode_advance_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(lens, batch, capacity);
     return cudaGetLastError();
 }
 

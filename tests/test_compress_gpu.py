@@ -232,6 +232,32 @@ def test_gemm_in_place_equals_fresh_copy(ctx):
     assert torch.equal(k, k2) and torch.equal(v, v2)
 
 
+def test_permuted_strides_layer_outermost(ctx):
+    """A cache stored layer-major ([layers, batch, heads, tokens, dim] in memory, presented as
+    [batch, layers, ...]): compression, append and decode attention must follow the strides."""
+    B, Ly, H, cap = 3, 2, 2, 300
+    w = small(cap=cap, dtype=torch.bfloat16, sink=4, outliers=2, B=B, Ly=Ly, H=H)
+    k0, v0 = synth.make_cache(w, "cuda")
+    k = k0.permute(1, 0, 2, 3, 4).contiguous().permute(1, 0, 2, 3, 4)   # same values, layer-major storage
+    v = v0.permute(1, 0, 2, 3, 4).contiguous().permute(1, 0, 2, 3, 4)
+    assert k.stride(1) > k.stride(0) and torch.equal(k, k0)
+    for variant in (fk.GEMM, fk.SIMT):
+        ka, va, kb, vb = k.clone(memory_format=torch.preserve_format), v.clone(memory_format=torch.preserve_format), k0.clone(), v0.clone()
+        assert ka.stride() == k.stride()
+        ctx.set_variant(variant)
+        ctx.compress(ka, va, cap, 148, 4)
+        ctx.compress(kb, vb, cap, 148, 4)
+        assert torch.equal(ka, kb) and torch.equal(va, vb)
+    ctx.set_variant(fk.AUTO)
+    nk = torch.randn(B, Ly, H, 7, 128, device="cuda").to(torch.bfloat16)
+    ka, kb = k.clone(memory_format=torch.preserve_format), k0.clone()
+    va, vb = v.clone(memory_format=torch.preserve_format), v0.clone()
+    assert ctx.append(ka, va, nk, nk, [10, 200, 293]) == ctx.append(kb, vb, nk, nk, [10, 200, 293])
+    assert torch.equal(ka, kb) and torch.equal(va, vb)
+    q = torch.randn(B, H, 128, device="cuda").to(torch.bfloat16)
+    assert torch.equal(ctx.attend_decode(ka, va, 1, q, [17, 207, 300]), ctx.attend_decode(kb, vb, 1, q, [17, 207, 300]))
+
+
 # ---- other retention patterns: retaining ratios 0.25 / 0.75 / 1 %, and another band of components
 @pytest.mark.parametrize("n_in,kept", [(4092, 1023), (4092, 3069), (4092, 40), (1000, 10)])
 def test_other_retaining_ratios_gemm(ctx, n_in, kept):

@@ -159,10 +159,10 @@ bool fdct_applicable(const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 }
 
 // Variant table, from measurements on B200 (7B shape, 2048 matrices): at 4096 -> 2048 bf16 the
-// tensor-core projection takes 2.96 ms and the fast transform 5.73 ms, so bf16 caches with
-// head_dim 128 go to the tensor cores whenever a tile can be filled; the fast transform serves
-// the power-of-two shapes the tensor-core path does not take (fp32 caches, other head sizes);
-// everything else runs as a projection on the CUDA cores.
+// tensor-core projection takes 2.36 ms (fold pass included) and the fast transform 4.63 ms, so
+// bf16 caches with head_dim 128 go to the tensor cores whenever a tile can be filled; the fast
+// transform serves the power-of-two shapes the tensor-core path does not take (fp32 caches, other
+// head sizes); everything else runs as a projection on the CUDA cores.
 int32_t resolve(const freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 {
     const bool g = gemm_applicable(l, n_in, n_keep), f = fdct_applicable(l, n_in, n_keep);

@@ -17,9 +17,12 @@
 // One CTA owns 8192 complex points = P channel pairs of one matrix (P = 8192 / N), keeps them in
 // shared memory for the whole chain and writes the L output rows over the input rows of its own
 // channels: no other CTA touches those columns, so the transform is in place in global memory
-// with no scratch.  FFT passes are Stockham radix-16 (remainder 8/4/2) butterflies held in
-// registers; a thread reads all its inputs, the CTA synchronises, then it writes.  Indices are
-// padded by one element per 16 so the stride-16 writes of the first pass are conflict-free.
+// with no scratch.  Both FFTs run in place in shared memory, one radix-16 (8/4/2 for the odd
+// factor) butterfly at a time per thread, held in registers: the forward one as decimation in
+// time on digit-reversed input -- the load phase puts every element where that order wants it --
+// the inverse one as decimation in frequency, whose digit-reversed output the store phase reads
+// back in row order.  Twiddles come from an fp64-built table through the read-only cache.
+// Indices are padded (see pad()) so that the passes meet few shared-memory bank conflicts.
 #include <cuda.h>
 
 #include "fdct.cuh"
@@ -29,9 +32,10 @@ namespace {
 
 constexpr int POINTS = 8192;  // complex points per CTA
 constexpr int THREADS = 256;
-constexpr int PPT = POINTS / THREADS;  // 32 points per thread in a forward pass
 
-__device__ __forceinline__ int pad(int i) { return i + (i >> 4); }
+// One extra element per 16 and one more per 256: elements 1, 16 or 256 apart (the strides of the
+// passes and of the digit-reversed placement) then fall into different shared-memory banks.
+__host__ __device__ __forceinline__ int pad(int i) { return i + (i >> 4) + (i >> 8); }
 
 __device__ __forceinline__ float2 cmul(float2 a, float2 b)
 {
@@ -90,76 +94,133 @@ struct SmallFft<1, INV> {
     static __device__ __forceinline__ void run(float2 (&)[1]) {}
 };
 
-// One Stockham pass of radix R over `pairs` sequences of length n stored at s[pair * ps + pad(i)].
-// Butterfly j (of n/R per sequence) reads x[j + r n/R], multiplies by w^(r k) with k = j mod ns and
-// w = exp(-+ 2 pi i / (ns R)), transforms, and writes y[(j - k) R + k + r ns].
-template <int R, int B, bool INV>
-__device__ __forceinline__ void fft_pass(float2* s, int log_n, int ps, int pairs, int log_ns, const float2* __restrict__ W,
-                                         int log_table, int tid)
+// One transform is a sequence of in-place passes, each with a radix R = 2^log_r and a stride
+// S = 2^log_s (the product of the radices of the passes below it): radix-16 passes with strides
+// 1, 16, 256, ..., then, when log2 of the length is not a multiple of 4, one pass of radix 8, 4 or 2
+// on top.  (Lengths are at least 16, so pass 0 always has radix 16.)
+struct Passes {
+    int32_t count;
+    int32_t log_r[4], log_s[4];
+};
+
+// Where element n of the natural order sits in the digit-reversed order that goes with `passes`:
+// the lowest digit of n (radix of the last pass) selects the block of the largest stride, and so on.
+__device__ __forceinline__ int digit_pos(int n, const Passes& ps)
 {
-    float2 v[B][R];
-    int dst[B];  // pair << 20 | first output index; -1 when this slot has no butterfly
-    constexpr int log_r = R == 16 ? 4 : R == 8 ? 3 : R == 4 ? 2 : 1;
-    const int log_bf = log_n - log_r;  // butterflies per sequence
-    const int total = pairs << log_bf;
-    const int span = 1 << log_bf, ns = 1 << log_ns;
+    int pos = 0;
 #pragma unroll
-    for (int b = 0; b < B; ++b) {
-        const int g = tid + b * THREADS;
-        dst[b] = -1;
-        if (g < total) {
-            const int pair = g >> log_bf, j = g & (span - 1), k = j & (ns - 1);
-            const float2* x = s + pair * ps;
-#pragma unroll
-            for (int r = 0; r < R; ++r) v[b][r] = x[pad(j + r * span)];
-            if (log_ns > 0) {
-                float2 w1 = W[k << (log_table - log_r - log_ns)];  // exp(-2 pi i k / (ns R))
-                if (INV) w1.y = -w1.y;
-                float2 w = w1;
-#pragma unroll
-                for (int r = 1; r < R; ++r) {
-                    v[b][r] = cmul(v[b][r], w);
-                    if (r + 1 < R) w = cmul(w, w1);
-                }
-            }
-            SmallFft<R, INV>::run(v[b]);
-            dst[b] = (pair << 20) | ((j - k) * R + k);
+    for (int p = 3; p >= 0; --p) {
+        if (p < ps.count) {
+            pos += (n & ((1 << ps.log_r[p]) - 1)) << ps.log_s[p];
+            n >>= ps.log_r[p];
         }
     }
-    __syncthreads();
-#pragma unroll
-    for (int b = 0; b < B; ++b) {
-        if (dst[b] >= 0) {
-            float2* y = s + (dst[b] >> 20) * ps;
-            const int j0 = dst[b] & ((1 << 20) - 1);
-#pragma unroll
-            for (int r = 0; r < R; ++r) y[pad(j0 + r * ns)] = v[b][r];
+    return pos;
+}
+
+// v[q] *= w^q, q = 1 .. R-1.
+template <int R>
+__device__ __forceinline__ void twiddle_all(float2 (&v)[R], float2 w1)
+{
+    v[1] = cmul(v[1], w1);
+    if constexpr (R >= 4) {
+        const float2 w2 = cmul(w1, w1), w3 = cmul(w2, w1);
+        v[2] = cmul(v[2], w2);
+        v[3] = cmul(v[3], w3);
+        if constexpr (R >= 8) {
+            const float2 w4 = cmul(w2, w2);
+            v[4] = cmul(v[4], w4);
+            v[5] = cmul(v[5], cmul(w4, w1));
+            v[6] = cmul(v[6], cmul(w4, w2));
+            v[7] = cmul(v[7], cmul(w4, w3));
+            if constexpr (R >= 16) {
+                const float2 w8 = cmul(w4, w4), w12 = cmul(w8, w4);
+                v[8] = cmul(v[8], w8);
+                v[9] = cmul(v[9], cmul(w8, w1));
+                v[10] = cmul(v[10], cmul(w8, w2));
+                v[11] = cmul(v[11], cmul(w8, w3));
+                v[12] = cmul(v[12], w12);
+                v[13] = cmul(v[13], cmul(w12, w1));
+                v[14] = cmul(v[14], cmul(w12, w2));
+                v[15] = cmul(v[15], cmul(w12, w3));
+            }
         }
+    }
+}
+
+// One in-place pass over `pairs` sequences of 2^log_n points stored at s[pair * stride + pad(i)].
+// Butterfly g of a sequence (2^(log_n - log_r) of them) works on the R elements base + q S,
+// base = (g / S) S R + k, k = g mod S.  A thread does its butterflies one after the other.
+//   forward (decimation in time, input digit-reversed, output natural):
+//     element q is multiplied by w^(q k), w = exp(-2 pi i / (S R)), then the R-point DFT;
+//   inverse (decimation in frequency, input natural, output digit-reversed):
+//     the R-point inverse DFT, then output r is multiplied by conj(w)^(r k).
+// W[j] = exp(-2 pi i j / 2^log_table).
+// The stride is 1, 16, 256 or 4096 (see make_passes), for which the padded position of element q
+// is pad(base) + q * STEP with a constant STEP: S = 1: consecutive (base is a multiple of R);
+// S = 16: base + 16 q stays inside one group of 256, so only the per-16 padding grows, by one per q;
+// S a multiple of 256: both paddings grow by whole amounts.
+template <int R, int LOG_S, bool INV>
+__device__ __forceinline__ void fft_pass(float2* s, int log_n, int seq_stride, int pairs, const float2* __restrict__ W,
+                                         int log_table, int tid)
+{
+    constexpr int log_r = R == 16 ? 4 : R == 8 ? 3 : R == 4 ? 2 : 1;
+    constexpr int S = 1 << LOG_S;
+    constexpr int STEP = LOG_S == 0 ? 1 : LOG_S == 4 ? 17 : S + (S >> 4) + (S >> 8);
+    const int log_bf = log_n - log_r;  // butterflies per sequence
+    const int total = pairs << log_bf;
+    const int tw_shift = log_table - LOG_S - log_r;
+    for (int g = tid; g < total; g += THREADS) {
+        const int pair = g >> log_bf, j = g & ((1 << log_bf) - 1), k = j & (S - 1);
+        float2* x = s + pair * seq_stride + pad(((j >> LOG_S) << (LOG_S + log_r)) + k);
+        float2 v[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) v[q] = x[q * STEP];
+        if constexpr (LOG_S > 0) {
+            // w^q for q = 1 .. R-1 from one table entry: w^2 and w^3 by products, the rest as
+            // w^(4a+b) = (w^4)^a w^b, so that no power is more than three products away from the table
+            float2 w1 = __ldg(W + (k << tw_shift));
+            if (INV) w1.y = -w1.y;
+            if (!INV) twiddle_all<R>(v, w1);
+            SmallFft<R, INV>::run(v);
+            if (INV) twiddle_all<R>(v, w1);
+        } else {
+            SmallFft<R, INV>::run(v);
+        }
+#pragma unroll
+        for (int q = 0; q < R; ++q) x[q * STEP] = v[q];
     }
     __syncthreads();
 }
 
-// All passes of one transform of length 2^log_n over `pairs` sequences.  PPT_ = points per thread
-// (32 forward, fewer for the shorter inverse); a radix-R pass gives each thread max(1, PPT_/R)
-// butterflies, guarded by the butterfly count.
-template <bool INV, int PPT_>
-__device__ __forceinline__ void fft_all(float2* s, int log_n, int ps, int pairs, const float2* __restrict__ W,
-                                        int log_table, int tid)
+template <int LOG_S, bool INV>
+__device__ __forceinline__ void fft_pass_radix(int log_r, float2* s, int log_n, int seq_stride, int pairs,
+                                               const float2* __restrict__ W, int log_table, int tid)
 {
-    int log_ns = 0, left = log_n;
-    while (left > 0) {
-        if (left >= 4) {
-            fft_pass<16, (PPT_ >= 16 ? PPT_ / 16 : 1), INV>(s, log_n, ps, pairs, log_ns, W, log_table, tid);
-            log_ns += 4, left -= 4;
-        } else if (left == 3) {
-            fft_pass<8, (PPT_ >= 8 ? PPT_ / 8 : 1), INV>(s, log_n, ps, pairs, log_ns, W, log_table, tid);
-            log_ns += 3, left -= 3;
-        } else if (left == 2) {
-            fft_pass<4, (PPT_ >= 4 ? PPT_ / 4 : 1), INV>(s, log_n, ps, pairs, log_ns, W, log_table, tid);
-            log_ns += 2, left -= 2;
-        } else {
-            fft_pass<2, (PPT_ >= 2 ? PPT_ / 2 : 1), INV>(s, log_n, ps, pairs, log_ns, W, log_table, tid);
-            log_ns += 1, left -= 1;
+    switch (log_r) {
+        case 4: fft_pass<16, LOG_S, INV>(s, log_n, seq_stride, pairs, W, log_table, tid); break;
+        case 3: fft_pass<8, LOG_S, INV>(s, log_n, seq_stride, pairs, W, log_table, tid); break;
+        case 2: fft_pass<4, LOG_S, INV>(s, log_n, seq_stride, pairs, W, log_table, tid); break;
+        default: fft_pass<2, LOG_S, INV>(s, log_n, seq_stride, pairs, W, log_table, tid); break;
+    }
+}
+
+// All passes of one transform, in the order the direction needs: forward from stride 1 up,
+// inverse from the largest stride down.
+template <bool INV>
+__device__ __forceinline__ void fft_all(float2* s, int log_n, int seq_stride, int pairs, const Passes& ps,
+                                        const float2* __restrict__ W, int log_table, int tid)
+{
+    // (constant indices into the pass list: it lives in the kernel's parameter space)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int p = INV ? 3 - i : i;
+        if (p >= ps.count) continue;
+        switch (ps.log_s[p]) {
+            case 0: fft_pass<16, 0, INV>(s, log_n, seq_stride, pairs, W, log_table, tid); break;  // stride 1 is always radix 16
+            case 4: fft_pass_radix<4, INV>(ps.log_r[p], s, log_n, seq_stride, pairs, W, log_table, tid); break;
+            case 8: fft_pass_radix<8, INV>(ps.log_r[p], s, log_n, seq_stride, pairs, W, log_table, tid); break;
+            default: fft_pass_radix<12, INV>(ps.log_r[p], s, log_n, seq_stride, pairs, W, log_table, tid); break;
         }
     }
 }
@@ -177,11 +238,36 @@ __device__ __forceinline__ float2 load_pair<__nv_bfloat16>(const __nv_bfloat16* 
     const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
     return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
 }
+// Two neighbouring pairs (four channels) with one load.
+__device__ __forceinline__ void load_two_pairs(const float* p, float2& a, float2& b)
+{
+    const float4 u = *reinterpret_cast<const float4*>(p);
+    a = make_float2(u.x, u.y);
+    b = make_float2(u.z, u.w);
+}
+__device__ __forceinline__ void load_two_pairs(const __nv_bfloat16* p, float2& a, float2& b)
+{
+    const uint2 u = *reinterpret_cast<const uint2*>(p);
+    a = make_float2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+    b = make_float2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+}
 __device__ __forceinline__ void store_pair(float* p, float2 v) { *reinterpret_cast<float2*>(p) = v; }
 __device__ __forceinline__ void store_pair(__nv_bfloat16* p, float2 v)
 {
     const __nv_bfloat162 b = __floats2bfloat162_rn(v.x, v.y);
     *reinterpret_cast<uint32_t*>(p) = *reinterpret_cast<const uint32_t*>(&b);
+}
+__device__ __forceinline__ void store_two_pairs(float* p, float2 a, float2 b)
+{
+    *reinterpret_cast<float4*>(p) = make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ void store_two_pairs(__nv_bfloat16* p, float2 a, float2 b)
+{
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(b.x, b.y);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t*>(&lo);
+    u.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = u;
 }
 
 struct FdctParams {
@@ -189,37 +275,48 @@ struct FdctParams {
     int32_t log_pairs;        // P = 2^log_pairs channel pairs per CTA (P * N = POINTS)
     int32_t groups_per_mat;   // head_dim / (2 P)
     int32_t sink;
+    Passes fwd, inv;          // pass lists of the N-point and of the L-point transform
     const float2* W;          // exp(-2 pi i q / N), q < N
     const float2* phi;        // exp(-i pi t / (2N)) / N, t <= L
     const float2* psi;        // exp(+i pi t / (2L)) / 2, t <= L
 };
 
 template <typename T>
-__global__ void __launch_bounds__(THREADS, 2) fdct_kernel(CacheView view, FdctParams prm)
+__global__ void __launch_bounds__(THREADS, 3) fdct_kernel(CacheView view, FdctParams prm)
 {
     extern __shared__ float2 s[];
     const int tid = threadIdx.x;
     const int N = 1 << prm.log_n, L = 1 << prm.log_l, P = 1 << prm.log_pairs;
-    const int ps = pad(N) + 1;  // sequence stride in shared memory (odd multiple keeps pairs on different banks)
+    const int ps = pad(N) + 1;  // sequence stride in shared memory
 
     const int32_t mat = blockIdx.x / prm.groups_per_mat, group = blockIdx.x % prm.groups_per_mat;
     const int32_t tensor = mat / view.mats_per_tensor;
     T* x = static_cast<T*>(tensor_base(view, tensor)) + matrix_offset(view, mat % view.mats_per_tensor) +
            (int64_t)prm.sink * view.stride_token + group * 2 * P;
 
-    // 1. load and reorder: row m -> v index m/2 (m even) or N-1-(m-1)/2 (m odd)
-#pragma unroll 4
-    for (int i = 0; i < PPT; ++i) {
-        const int idx = tid + i * THREADS;
-        const int m = idx >> prm.log_pairs, p = idx & (P - 1);
-        const float2 w = load_pair<T>(x + (int64_t)m * view.stride_token + 2 * p);
-        const int vi = (m & 1) ? N - 1 - (m >> 1) : (m >> 1);
-        s[p * ps + pad(vi)] = w;
+    // 1. load, reorder (row m -> v index m/2 for even m, N-1-(m-1)/2 for odd m) and place every
+    //    element where the in-place forward transform wants it (digit-reversed)
+    if (P >= 2) {
+        const int half = P >> 1, log_half = prm.log_pairs - 1;
+        for (int idx = tid; idx < (N << log_half); idx += THREADS) {
+            const int m = idx >> log_half, p2 = idx & (half - 1);
+            float2 a, b;
+            load_two_pairs(x + (int64_t)m * view.stride_token + 4 * p2, a, b);
+            const int vi = (m & 1) ? N - 1 - (m >> 1) : (m >> 1);
+            const int at = pad(digit_pos(vi, prm.fwd));
+            s[(2 * p2) * ps + at] = a;
+            s[(2 * p2 + 1) * ps + at] = b;
+        }
+    } else {
+        for (int m = tid; m < N; m += THREADS) {
+            const int vi = (m & 1) ? N - 1 - (m >> 1) : (m >> 1);
+            s[pad(digit_pos(vi, prm.fwd))] = load_pair<T>(x + (int64_t)m * view.stride_token);
+        }
     }
     __syncthreads();
 
-    // 2. forward FFT of length N on every pair
-    fft_all<false, PPT>(s, prm.log_n, ps, P, prm.W, prm.log_n, tid);
+    // 2. forward FFT of length N on every pair (natural order out)
+    fft_all<false>(s, prm.log_n, ps, P, prm.fwd, prm.W, prm.log_n, tid);
 
     // 3-4. spectrum of the DCT, truncation, and the pre-twiddle of the inverse, in place in [0, L)
     {
@@ -230,12 +327,12 @@ __global__ void __launch_bounds__(THREADS, 2) fdct_kernel(CacheView view, FdctPa
             const int p = idx >> log_half, t = (idx & (half - 1)) + 1, u = L - t;
             float2* q = s + p * ps;
             const float2 vt = q[pad(t)], vnt = q[pad(N - t)], vu = q[pad(u)], vnu = q[pad(N - u)];
-            const float2 ft = prm.phi[t], fu = prm.phi[u];
+            const float2 ft = __ldg(prm.phi + t), fu = __ldg(prm.phi + u);
             const float2 gt = cadd(cmul(ft, vt), cmul(conjf2(ft), vnt));
             const float2 gu = cadd(cmul(fu, vu), cmul(conjf2(fu), vnu));
             // U_t = psi_t (g_t - i g_u), U_u = psi_u (g_u - i g_t);  -i (a + ib) = b - ia
-            const float2 ut = cmul(prm.psi[t], make_float2(gt.x + gu.y, gt.y - gu.x));
-            const float2 uu = cmul(prm.psi[u], make_float2(gu.x + gt.y, gu.y - gt.x));
+            const float2 ut = cmul(__ldg(prm.psi + t), make_float2(gt.x + gu.y, gt.y - gu.x));
+            const float2 uu = cmul(__ldg(prm.psi + u), make_float2(gu.x + gt.y, gu.y - gt.x));
             q[pad(t)] = ut;
             q[pad(u)] = uu;
         }
@@ -247,20 +344,22 @@ __global__ void __launch_bounds__(THREADS, 2) fdct_kernel(CacheView view, FdctPa
     }
     __syncthreads();
 
-    // 5. inverse FFT of length L, then un-reorder and store over rows [sink, sink + L)
-    switch (prm.log_n - prm.log_l) {  // points per thread of the inverse = 32 L / N
-        case 1: fft_all<true, 16>(s, prm.log_l, ps, P, prm.W, prm.log_n, tid); break;
-        case 2: fft_all<true, 8>(s, prm.log_l, ps, P, prm.W, prm.log_n, tid); break;
-        case 3: fft_all<true, 4>(s, prm.log_l, ps, P, prm.W, prm.log_n, tid); break;
-        case 4: fft_all<true, 2>(s, prm.log_l, ps, P, prm.W, prm.log_n, tid); break;
-        default: fft_all<true, 1>(s, prm.log_l, ps, P, prm.W, prm.log_n, tid); break;
-    }
+    // 5. inverse FFT of length L (digit-reversed order out), then un-reorder and store over rows [sink, sink + L)
+    fft_all<true>(s, prm.log_l, ps, P, prm.inv, prm.W, prm.log_n, tid);
 
-    const int out_items = P << prm.log_l;
-    for (int idx = tid; idx < out_items; idx += THREADS) {
-        const int m = idx >> prm.log_pairs, p = idx & (P - 1);
-        const int ri = (m & 1) ? L - 1 - (m >> 1) : (m >> 1);
-        store_pair(x + (int64_t)m * view.stride_token + 2 * p, s[p * ps + pad(ri)]);
+    if (P >= 2) {
+        const int half = P >> 1, log_half = prm.log_pairs - 1;
+        for (int idx = tid; idx < (L << log_half); idx += THREADS) {
+            const int m = idx >> log_half, p2 = idx & (half - 1);
+            const int ri = (m & 1) ? L - 1 - (m >> 1) : (m >> 1);
+            const int at = pad(digit_pos(ri, prm.inv));
+            store_two_pairs(x + (int64_t)m * view.stride_token + 4 * p2, s[(2 * p2) * ps + at], s[(2 * p2 + 1) * ps + at]);
+        }
+    } else {
+        for (int m = tid; m < L; m += THREADS) {
+            const int ri = (m & 1) ? L - 1 - (m >> 1) : (m >> 1);
+            store_pair(x + (int64_t)m * view.stride_token, s[pad(digit_pos(ri, prm.inv))]);
+        }
     }
 }
 
@@ -289,10 +388,26 @@ int ilog2(int32_t x)
     return l;
 }
 
+Passes make_passes(int log_len)
+{
+    Passes ps = {};
+    int log_s = 0;
+    for (int i = 0; i < log_len / 4; ++i) {
+        ps.log_r[ps.count] = 4;
+        ps.log_s[ps.count++] = log_s;
+        log_s += 4;
+    }
+    if (log_len % 4) {
+        ps.log_r[ps.count] = log_len % 4;
+        ps.log_s[ps.count++] = log_s;
+    }
+    return ps;
+}
+
 size_t smem_bytes(int32_t N)
 {
     const int P = POINTS / N;
-    return (size_t)P * ((N + (N >> 4)) + 1) * sizeof(float2);
+    return (size_t)P * (pad(N) + 1) * sizeof(float2);
 }
 
 }  // namespace
@@ -355,6 +470,8 @@ cudaError_t launch_fdct(const CacheView& view, int32_t dtype, int32_t n_mat, con
     prm.log_pairs = ilog2(P);
     prm.groups_per_mat = view.head_dim / (2 * P);
     prm.sink = sink;
+    prm.fwd = make_passes(prm.log_n);
+    prm.inv = make_passes(prm.log_l);
     prm.W = plan.twiddle;
     prm.phi = plan.twiddle + plan.n_in;
     prm.psi = prm.phi + plan.n_keep + 1;

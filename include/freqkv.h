@@ -15,7 +15,10 @@
  *    Calls enqueue work on it and return without synchronising, unless stated otherwise.
  *  - Every function returns a freqkv_status; on any status other than FREQKV_OK nothing was
  *    enqueued and no caller memory was modified.  No C++ exception crosses the boundary.
- *  - A context belongs to one device and must not be used from two threads at once.
+ *  - A context belongs to one device and must not be used from two threads at once.  Its work
+ *    areas are shared by its calls: a call enqueued on another stream than the previous one first
+ *    waits (on the device) for that one, so calls on one context never overlap on the GPU; use
+ *    one context per stream for concurrency.
  *  - There is no CPU fallback: without a CUDA device freqkv_create fails.
  */
 #ifndef FREQKV_H_

@@ -32,6 +32,11 @@ struct freqkv_ctx {
     int32_t* status_dev = nullptr;
     GemmState gemm;
     std::string last_error;
+    // Work areas (fold scratch, staging, attention partials) are shared by all calls on this
+    // context: a call on another stream than the previous one first waits for that one's work.
+    cudaEvent_t work_done = nullptr;
+    cudaStream_t work_stream = nullptr;
+    bool work_recorded = false;
     // instrumentation
     bool timing = false;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> pending, spare;
@@ -70,6 +75,16 @@ struct DeviceGuard {
     }
 };
 
+// Orders the calls that use the context's work areas: on entry the caller's stream waits for the
+// previous such call if that one ran on a different stream; on exit the end of this call's work
+// is recorded.  (Calls on one stream are ordered anyway and pay nothing.)
+struct WorkOrder {
+    freqkv_ctx* ctx;
+    cudaStream_t stream;
+    WorkOrder(freqkv_ctx* c, cudaStream_t s);
+    ~WorkOrder();
+};
+
 freqkv_status cuda_fail(freqkv_ctx* ctx, cudaError_t e, const char* where)
 {
     if (ctx) ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
@@ -82,6 +97,26 @@ freqkv_status cuda_fail(freqkv_ctx* ctx, cudaError_t e, const char* where)
         const cudaError_t e__ = (call);                                    \
         if (e__ != cudaSuccess) return cuda_fail((ctx), e__, #call);       \
     } while (0)
+
+WorkOrder::WorkOrder(freqkv_ctx* c, cudaStream_t s) : ctx(c), stream(s)
+{
+    if (ctx->work_recorded && ctx->work_stream != stream) cudaStreamWaitEvent(stream, ctx->work_done, 0);
+}
+
+WorkOrder::~WorkOrder()
+{
+    if (!ctx->work_done && cudaEventCreateWithFlags(&ctx->work_done, cudaEventDisableTiming) != cudaSuccess) {
+        ctx->work_done = nullptr;
+        cudaGetLastError();
+        return;
+    }
+    if (cudaEventRecord(ctx->work_done, stream) == cudaSuccess) {
+        ctx->work_stream = stream;
+        ctx->work_recorded = true;
+    } else {
+        cudaGetLastError();
+    }
+}
 
 int64_t span_elements(const freqkv_layout& l)
 {
@@ -441,6 +476,7 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     for (int i = 0; i < 2; ++i)
         if (ctx->stage[i]) cudaFree(ctx->stage[i]);
+    if (ctx->work_done) cudaEventDestroy(ctx->work_done);
     if (ctx->rope_table) cudaFree(ctx->rope_table);
     if (ctx->attend_partial) cudaFree(ctx->attend_partial);
     for (int i = 0; i < 3; ++i)
@@ -543,6 +579,7 @@ freqkv_status freqkv_compress(freqkv_ctx* ctx, const freqkv_layout* layout, void
     if (variant < 0) return FREQKV_ERR_UNSUPPORTED;
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
+    WorkOrder order(ctx, static_cast<cudaStream_t>(cuda_stream));
     return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
                           static_cast<cudaStream_t>(cuda_stream));
 }
@@ -564,6 +601,7 @@ freqkv_status freqkv_compress_band(freqkv_ctx* ctx, const freqkv_layout* layout,
     if (variant < 0) return FREQKV_ERR_UNSUPPORTED;
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
+    WorkOrder order(ctx, static_cast<cudaStream_t>(cuda_stream));
     return compress_group(ctx, *layout, k, v, 0, layout->batch, n_in, kept_len, sink, variant,
                           static_cast<cudaStream_t>(cuda_stream), first_component);
 }
@@ -582,6 +620,7 @@ freqkv_status freqkv_power_spectrum(freqkv_ctx* ctx, const freqkv_layout* layout
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    WorkOrder order(ctx, stream);
     Basis basis;
     st = get_basis(ctx, n_in, n_in, kDctRows, false, true, stream, &basis);
     if (st != FREQKV_OK) return st;
@@ -624,6 +663,7 @@ freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layou
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    WorkOrder order(ctx, stream);
     // Sequences are grouped by runs of equal (length, kept length); each run is one group.
     for (int32_t b = 0; b < layout->batch;) {
         int32_t e = b + 1;
@@ -673,6 +713,7 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    WorkOrder order(ctx, stream);  // its end is recorded after the caller's stream has joined the pipeline's tail
     const size_t elt = dtype_size(l.dtype);
     const size_t bytes = (size_t)span_elements(l) * elt;
     if (bytes > ctx->stage_bytes) {
@@ -788,6 +829,7 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    WorkOrder order(ctx, stream);
     if (scale <= 0.f) scale = 1.0f / sqrtf((float)l.head_dim);
     int32_t max_len = 0;
     for (int32_t b = 0; b < l.batch; ++b) max_len = std::max(max_len, lens[b]);
@@ -928,6 +970,7 @@ freqkv_status freqkv_decode_graph_launch(freqkv_decode_graph* graph, void* cuda_
     if (!graph || !graph->exec) return FREQKV_ERR_INVALID_ARG;
     DeviceGuard g(graph->ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
+    WorkOrder order(graph->ctx, static_cast<cudaStream_t>(cuda_stream));  // the graph's kernels use the context's scratch
     FREQKV_CUDA(graph->ctx, cudaGraphLaunch(graph->exec, static_cast<cudaStream_t>(cuda_stream)));
     graph->ctx->kernels_launched += 3;  // trigger, append, advance (the compression adds 3 when it runs)
     return FREQKV_OK;

@@ -232,6 +232,29 @@ def test_gemm_in_place_equals_fresh_copy(ctx):
     assert torch.equal(k, k2) and torch.equal(v, v2)
 
 
+def test_calls_on_two_streams_share_one_context_safely(ctx):
+    """The context's scratch is shared: calls enqueued on different streams without any host
+    synchronisation must still give the results of running them one after the other."""
+    w = small(cap=1100, dtype=torch.bfloat16, sink=4, outliers=2, B=1, Ly=4, H=8)
+    caches = [synth.make_cache(dataclasses.replace(w, seed=w.seed + i), "cuda") for i in range(4)]
+    want = []
+    ctx.set_variant(fk.GEMM)
+    for k, v in caches:
+        k2, v2 = k.clone(), v.clone()
+        ctx.compress(k2, v2, 1100, 548, 4)
+        want.append((k2, v2))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for i, (k, v) in enumerate(caches):
+        with torch.cuda.stream(streams[i % 2]):
+            ctx.compress(k, v, 1100, 548, 4, stream=streams[i % 2])
+    torch.cuda.synchronize()
+    ctx.set_variant(fk.AUTO)
+    assert ctx.last_device_status() == fk.OK
+    for (k, v), (k2, v2) in zip(caches, want):
+        assert torch.equal(k, k2) and torch.equal(v, v2)
+
+
 def test_permuted_strides_layer_outermost(ctx):
     """A cache stored layer-major ([layers, batch, heads, tokens, dim] in memory, presented as
     [batch, layers, ...]): compression, append and decode attention must follow the strides."""

@@ -288,13 +288,14 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
     const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
                     (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
     const int64_t row_bytes = view.stride_token * 2;
-    const uint32_t total = (uint32_t)job.n_half * 16u, stride = gridDim.y * blockDim.x;
+    const uint32_t total = (uint32_t)job.n_half * 16u;
     uint4* u_plane = job.dst + (int64_t)pt * 2 * total;
-    for (uint32_t i0 = blockIdx.y * blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+    // a block works on chunks of 1024 consecutive vectors (64 rows and their 64 mirror rows)
+    for (uint32_t c0 = blockIdx.y * 1024u; c0 < total; c0 += gridDim.y * 1024u) {
         uint4 a[4], b[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint32_t i = i0 + j * stride;
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
             if (i < total) {
                 const int32_t n = (int32_t)(i >> 4), nr = job.n_in - 1 - n;
                 a[j] = __ldcs(reinterpret_cast<const uint4*>(x + n * row_bytes) + (i & 15u));
@@ -303,7 +304,7 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint32_t i = i0 + j * stride;
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
             if (i < total) {
                 const int32_t n = (int32_t)(i >> 4);
                 uint4 u, v;

@@ -45,7 +45,8 @@ typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
 /* Which kernel family executes the compression.
  *   GEMM  the DCT-II -> truncate -> IDCT -> rescale chain folded into one precomputed
  *         kept_len x n_in projection basis and run on the tcgen05 tensor cores (bf16 caches,
- *         head_dim 128 only);
+ *         head_dim 128 only); halved by the even/odd symmetry of the cosines after a fold pass
+ *         over the cache, or, for kept_len <= 256, straight from the cache without that pass;
  *   FDCT  fast-transform kernel (power-of-two n_in and kept_len only);
  *   SIMT  the same projection on the fp32 CUDA cores (any shape; the only path for fp32
  *         caches of non-power-of-two length);

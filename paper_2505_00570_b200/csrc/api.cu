@@ -217,6 +217,7 @@ void free_bases(freqkv_ctx* ctx)
     for (auto& kv : ctx->bases) {
         if (kv.second.f32) cudaFree(kv.second.f32);
         if (kv.second.fold) cudaFree(kv.second.fold);
+        if (kv.second.dense) cudaFree(kv.second.dense);
     }
     ctx->bases.clear();
     ctx->basis_bytes = 0;
@@ -231,8 +232,10 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
     Basis b;
     auto it = ctx->bases.find(key);
     if (it != ctx->bases.end()) b = it->second;
-    const bool make_f32 = need_f32 && !b.f32, make_fold = need_fold && !b.fold;
-    if (make_f32 || make_fold) {
+    // the tensor-core path wants the folded pair, or, for few kept rows, the dense bf16 matrix
+    const bool direct = need_fold && first != kDctRows && gemm_is_direct(n_keep);
+    const bool make_f32 = need_f32 && !b.f32, make_fold = need_fold && !direct && !b.fold, make_dense = direct && !b.dense;
+    if (make_f32 || make_fold || make_dense) {
         auto shape = [&](Basis& x) {
             x.n_in = n_in;
             x.n_keep = n_keep;
@@ -241,11 +244,13 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
             x.rows_pad = (n_keep + 63) / 64 * 64;
             x.fold_ld = ((n_in + 1) / 2 + 63) / 64 * 64;
             x.fold_rows_pad = ((n_keep + 1) / 2 + 255) / 256 * 256;
+            x.dense_rows_pad = 256;
         };
         shape(b);
         const size_t elems = (size_t)b.ld * b.rows_pad;
         const size_t fold_elems = (size_t)2 * b.fold_ld * b.fold_rows_pad;
-        const size_t want = (make_f32 ? elems * 4 : 0) + (make_fold ? fold_elems * 2 : 0);
+        const size_t dense_elems = (size_t)256 * b.ld;
+        const size_t want = (make_f32 ? elems * 4 : 0) + (make_fold ? fold_elems * 2 : 0) + (make_dense ? dense_elems * 2 : 0);
         if (ctx->basis_bytes + want > kBasisBudgetBytes) {
             FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // bases may be in use by enqueued kernels
             free_bases(ctx);
@@ -254,8 +259,16 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
         }
         float* pf = nullptr;
         __nv_bfloat16* pb = nullptr;
+        __nv_bfloat16* pd = nullptr;
         if (need_f32 && !b.f32) FREQKV_CUDA(ctx, cudaMalloc(&pf, elems * 4));
-        if (need_fold && !b.fold) {
+        if (direct && !b.dense) {
+            const cudaError_t e = cudaMalloc(&pd, dense_elems * 2);
+            if (e != cudaSuccess) {
+                if (pf) cudaFree(pf);
+                return cuda_fail(ctx, e, "cudaMalloc(basis)");
+            }
+        }
+        if (need_fold && !direct && !b.fold) {
             const cudaError_t e = cudaMalloc(&pb, fold_elems * 2);
             if (e != cudaSuccess) {
                 if (pf) cudaFree(pf);
@@ -272,11 +285,17 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
                                   : launch_build_folded_basis(pb, n_in, n_keep, first, b.fold_ld, b.fold_rows_pad, stream);
             ctx->kernels_launched += 1;
         }
+        if (e == cudaSuccess && pd) {
+            e = launch_build_basis(nullptr, pd, n_in, n_keep, first, b.ld, 256, stream);
+            ctx->kernels_launched += 1;
+        }
         if (e != cudaSuccess) {
             if (pf) cudaFree(pf);
             if (pb) cudaFree(pb);
+            if (pd) cudaFree(pd);
             return cuda_fail(ctx, e, "build_basis");
         }
+        if (pd) { b.dense = pd; ctx->basis_bytes += dense_elems * 2; }
         if (pf) { b.f32 = pf; ctx->basis_bytes += elems * 4; }
         if (pb) { b.fold = pb; ctx->basis_bytes += fold_elems * 2; }
         ctx->bases[key] = b;
@@ -373,7 +392,10 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
         hooks.user = &timer;
         hooks.before = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->begin(); };
         hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
-        const cudaError_t e = launch_gemm(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
+        const cudaError_t e =
+            gemm_is_direct(n_keep)
+                ? launch_gemm_direct(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream)
+                : launch_gemm(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
         if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
         ctx->kernels_launched += ctx->gemm.kernels_last_call;
         return FREQKV_OK;
@@ -906,7 +928,7 @@ freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* l
     Basis basis;
     st = get_basis(ctx, n_in, kept_len, 0, false, true, cs, &basis);
     cudaError_t e = st == FREQKV_OK ? cudaStreamSynchronize(cs) : cudaSuccess;
-    if (st == FREQKV_OK && e == cudaSuccess) e = gemm_prepare(&ctx->gemm, l.batch * l.layers * l.kv_heads, basis, ctx->sm_count);
+    if (st == FREQKV_OK && e == cudaSuccess) e = gemm_prepare(&ctx->gemm, gemm_is_direct(kept_len) ? 0 : l.batch * l.layers * l.kv_heads, basis, ctx->sm_count);
     freqkv_decode_graph* dg = new (std::nothrow) freqkv_decode_graph();
     auto fail = [&](freqkv_status code, cudaError_t ce, const char* where) {
         if (ce != cudaSuccess) code = cuda_fail(ctx, ce, where);

@@ -43,6 +43,9 @@ struct Basis {
     // m < ceil(n_keep/2), n < ceil(n_in/2), bf16, two planes of fold_rows_pad x fold_ld (see basis.cu).
     __nv_bfloat16* fold = nullptr;
     int32_t fold_ld = 0, fold_rows_pad = 0;
+    // Tensor-core path for at most 256 kept rows: the whole P in bf16, dense_rows_pad (256) x ld.
+    __nv_bfloat16* dense = nullptr;
+    int32_t dense_rows_pad = 0;
 };
 
 // ---- kernel launchers (each returns the cudaError_t of its launch) ----

@@ -179,6 +179,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int32_t c0,
+                                            int32_t c1, int32_t c2, int32_t c3, int32_t c4)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor of tcgen05.mma: start address, leading and stride byte offsets
 // (all in 16-byte units), descriptor version 1, 128-byte swizzle.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
@@ -320,15 +329,25 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
     }
 }
 
-// SPECTRUM = false: the compression above.  SPECTRUM = true: the basis holds the even and the odd
-// rows of the plain N-point DCT-II instead of Pe and Po, so S and D are the components z_2m and
-// z_2m+1 themselves; the epilogue squares them, sums over the 128 channels of its tensor and adds
-// the sum to the power spectrum of its (layer, kv head).  Nothing is written to the cache.
-template <bool SPECTRUM>
+// MODE_FOLD: the compression above.
+// MODE_SPECTRUM: the basis holds the even and the odd rows of the plain N-point DCT-II instead of
+//   Pe and Po, so S and D are the components z_2m and z_2m+1 themselves; the epilogue squares them,
+//   sums over the 128 channels of its tensor and adds the sum to the power spectrum of its
+//   (layer, kv head).  Nothing is written to the cache.
+// MODE_DIRECT: for at most 256 kept rows (small retaining ratios) the fold pass would cost more
+//   than it saves: the basis is the plain L x N matrix P, the input slices come straight from the
+//   cache (map_x = K tensor, map_v = V tensor, 5-D maps over the non-sink rows), there is one
+//   accumulator and one tile per (batch, layer, kv_head).  The tile's rows are stored only after
+//   every slice of its matrices has been read, so writing in place is safe here too.
+constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2;
+
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_x,
-                   const CacheView view, const GemmParams prm)
+                   const __grid_constant__ CUtensorMap map_v, const CacheView view, const GemmParams prm)
 {
+    constexpr bool SPECTRUM = MODE == MODE_SPECTRUM;
+    constexpr int PHASES = MODE == MODE_DIRECT ? 1 : 2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
@@ -380,7 +399,10 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters) {
                 const int32_t pair_local = tile / prm.m_pairs;
                 const int32_t m0 = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM;
-                for (int eo = 0; eo < 2 && alive; ++eo) {
+                const int32_t pair = prm.pair0 + pair_local;  // direct mode: coordinates inside the cache tensor
+                const int32_t head = pair % view.kv_heads, layer = (pair / view.kv_heads) % view.layers,
+                              seq = pair / (view.kv_heads * view.layers);
+                for (int eo = 0; eo < PHASES && alive; ++eo) {
                     const int32_t plane = (pair_local * 2 + (int32_t)rank) * 2 + eo;  // rank 0: K channels, rank 1: V
                     for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
                         const int s = it % STAGES;
@@ -394,8 +416,14 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
                         const int32_t k0 = ks * BK;
                         tma_load_2d(stage, &map_p, leader_full, k0, eo * prm.basis_rows_pad + m0);
-                        tma_load_3d(stage + A_BYTES, &map_x, leader_full, 0, k0, plane);
-                        tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, &map_x, leader_full, 64, k0, plane);
+                        if constexpr (MODE == MODE_DIRECT) {
+                            const CUtensorMap* cache = rank ? &map_v : &map_x;
+                            tma_load_5d(stage + A_BYTES, cache, leader_full, 0, k0, head, layer, seq);
+                            tma_load_5d(stage + A_BYTES + B_CHUNK_BYTES, cache, leader_full, 64, k0, head, layer, seq);
+                        } else {
+                            tma_load_3d(stage + A_BYTES, &map_x, leader_full, 0, k0, plane);
+                            tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, &map_x, leader_full, 64, k0, plane);
+                        }
                     }
                 }
             }
@@ -410,7 +438,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             uint32_t it = 0, tile_no = 0;
             bool alive = true;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters, ++tile_no) {
-                for (int eo = 0; eo < 2 && alive; ++eo) {
+                for (int eo = 0; eo < PHASES && alive; ++eo) {
                     if (tile_no > 0) {  // both CTAs' epilogues must have read this accumulator of the last tile
                         if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT)) {
                             alive = false;
@@ -446,7 +474,32 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tensor * 128;
         const uint32_t leader_s_empty = cluster_addr(acc_empty_bar(0), 0), leader_d_empty = cluster_addr(acc_empty_bar(1), 0);
         uint32_t tile_no = 0;
-        if constexpr (SPECTRUM) {
+        if constexpr (MODE == MODE_DIRECT) {
+            for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
+                if (!mbar_wait(acc_full_bar(0), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const int32_t m = (int32_t)rank * BM + quarter * 32 + lane;
+                __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
+                                     matrix_offset(view, prm.pair0 + tile) + (int64_t)prm.sink * view.stride_token;
+                uint4* out = reinterpret_cast<uint4*>(mat + (int64_t)m * view.stride_token);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t y[16];
+                    tmem_ld16(lane_addr + c * 16, y);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (m < prm.n_keep) {
+                        uint32_t p[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) p[j] = pack_bf16(__uint_as_float(y[2 * j]), __uint_as_float(y[2 * j + 1]));
+                        out[2 * c] = make_uint4(p[0], p[1], p[2], p[3]);
+                        out[2 * c + 1] = make_uint4(p[4], p[5], p[6], p[7]);
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(leader_s_empty);
+            }
+        } else if constexpr (SPECTRUM) {
             for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
                 const int32_t pair = prm.pair0 + tile / prm.m_pairs;
                 const int32_t head = pair % view.kv_heads, layer = (pair / view.kv_heads) % view.layers;
@@ -597,7 +650,8 @@ bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_kee
 }
 
 // Everything a launch needs that is not a stream operation: kernel attributes, the count of
-// resident CTA pairs, the scratch buffer for `pairs` (batch, layer, kv_head) triples of this basis.
+// resident CTA pairs, the scratch buffer for `pairs` (batch, layer, kv_head) triples of this basis
+// (pairs = 0: none, the direct mode reads the cache itself).
 // launch_gemm calls it itself; a caller that must not allocate later (stream capture) calls it first.
 cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, int sm_count)
 {
@@ -607,9 +661,11 @@ cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, in
         return cudaErrorNotSupported;
     }
     if (!state->attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(freqkv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_FOLD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(freqkv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_SPECTRUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) {
             state->last_error = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -627,7 +683,7 @@ cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, in
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int n = 0;
-        const cudaError_t q = cudaOccupancyMaxActiveClusters(&n, freqkv_gemm_kernel<false>, &cfg);
+        const cudaError_t q = cudaOccupancyMaxActiveClusters(&n, freqkv_gemm_kernel<MODE_FOLD>, &cfg);
         if (q != cudaSuccess || n < 1) {
             state->last_error = "cudaOccupancyMaxActiveClusters: no CTA pair fits on this device";
             return q != cudaSuccess ? q : cudaErrorLaunchOutOfResources;
@@ -724,8 +780,8 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (hooks.before) hooks.before(hooks.user, stream);
-        e = spectrum ? cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<true>, map_p, map_x, view, prm)
-                     : cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<false>, map_p, map_x, view, prm);
+        e = spectrum ? cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_SPECTRUM>, map_p, map_x, map_x, view, prm)
+                     : cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_FOLD>, map_p, map_x, map_x, view, prm);
         if (hooks.after) hooks.after(hooks.user, stream);
         if (e != cudaSuccess) {
             state->last_error = "freqkv_gemm_kernel launch";
@@ -733,6 +789,89 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         }
         state->kernels_last_call += 2;
     }
+    return cudaSuccess;
+}
+
+// The non-sink rows of one cache tensor as a 5-D tensor (channel, token, kv_head, layer, batch).
+static bool encode_cache_map(CUtensorMap* map, const CacheView& view, int tensor, int32_t batch_count, int32_t n_in, int32_t sink)
+{
+    char* p = static_cast<char*>(tensor ? view.base[1] : view.base[0]) +
+              ((int64_t)view.batch0 * view.stride_batch + (int64_t)sink * view.stride_token) * 2;
+    const cuuint64_t dims[5] = {128, (cuuint64_t)n_in, (cuuint64_t)view.kv_heads, (cuuint64_t)view.layers,
+                                (cuuint64_t)batch_count};
+    // an axis of extent 1 is never stepped; give it a harmless stride
+    const cuuint64_t row = (cuuint64_t)view.stride_token * 2;
+    const cuuint64_t strides[4] = {row, view.kv_heads > 1 ? (cuuint64_t)view.stride_head * 2 : row,
+                                   view.layers > 1 ? (cuuint64_t)view.stride_layer * 2 : row,
+                                   batch_count > 1 ? (cuuint64_t)view.stride_batch * 2 : row};
+    const cuuint32_t box[5] = {64, BK, 1, 1, 1};
+    const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, p, dims, strides, box, elem,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool gemm_is_direct(int32_t n_keep) { return n_keep <= 2 * BM; }
+
+cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
+                               int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream)
+{
+    state->kernels_last_call = 0;
+    const cudaError_t prepared = gemm_prepare(state, 0, basis, sm_count);
+    if (prepared != cudaSuccess) return prepared;
+    const int32_t pairs = view.mats_per_tensor;
+    const int32_t batch_count = pairs / (view.layers * view.kv_heads);
+    CUtensorMap map_p, map_k, map_v;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)basis.ld, (cuuint64_t)basis.dense_rows_pad};
+        const cuuint64_t strides[1] = {(cuuint64_t)basis.ld * 2};
+        const cuuint32_t box[2] = {BK, BM};
+        const cuuint32_t elem[2] = {1, 1};
+        if (encode_fn()(&map_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, basis.dense, dims, strides, box, elem,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            state->last_error = "tensor map encoding rejected the basis";
+            return cudaErrorInvalidValue;
+        }
+    }
+    if (!encode_cache_map(&map_k, view, 0, batch_count, basis.n_in, sink) ||
+        !encode_cache_map(&map_v, view, 1, batch_count, basis.n_in, sink)) {
+        state->last_error = "tensor map encoding rejected this layout";
+        return cudaErrorInvalidValue;
+    }
+    GemmParams prm = {};
+    prm.n_keep = basis.n_keep;
+    prm.rows_half = basis.n_keep;
+    prm.basis_rows_pad = 0;
+    prm.pair0 = 0;
+    prm.pair_count = pairs;
+    prm.m_pairs = 1;
+    prm.k_steps = (basis.n_in + BK - 1) / BK;
+    prm.sink = sink;
+    prm.mirror_sign = 1;
+    prm.n_in = basis.n_in;
+    prm.status = status_dev;
+    const int clusters = std::min<int32_t>(pairs, state->max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (hooks.before) hooks.before(hooks.user, stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_DIRECT>, map_p, map_k, map_v, view, prm);
+    if (hooks.after) hooks.after(hooks.user, stream);
+    if (e != cudaSuccess) {
+        state->last_error = "freqkv_gemm_kernel launch";
+        return e;
+    }
+    state->kernels_last_call = 1;
     return cudaSuccess;
 }
 

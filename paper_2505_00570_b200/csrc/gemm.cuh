@@ -33,6 +33,10 @@ bool gemm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_kee
 cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink, int32_t* status_dev,
                         int sm_count, const LaunchHooks& hooks, cudaStream_t stream, const SpectrumOut* spectrum = nullptr);
 cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, int sm_count);
+// At most 256 kept rows: one tile per (batch, layer, kv_head), no fold pass, the dense basis (Basis::dense).
+bool gemm_is_direct(int32_t n_keep);
+cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
+                               int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 void gemm_release(GemmState* state);
 
 }  // namespace freqkv

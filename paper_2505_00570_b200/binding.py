@@ -110,13 +110,24 @@ def dtype_code(dtype: torch.dtype) -> int:
     raise FreqKVError(ERR_UNSUPPORTED, f"unsupported cache dtype {dtype}")
 
 
+_layout_cache: dict = {}
+
+
 def layout_of(t: torch.Tensor) -> Layout:
     """``freqkv_layout`` of a ``[batch, layers, kv_heads, capacity, head_dim]`` tensor (a view
-    with arbitrary strides is fine as long as head_dim is contiguous)."""
-    if t.dim() != 5 or t.stride(4) != 1:
-        raise FreqKVError(ERR_UNSUPPORTED, "cache must be [batch, layers, kv_heads, capacity, head_dim] with contiguous head_dim")
-    return Layout(dtype_code(t.dtype), t.shape[0], t.shape[1], t.shape[2], t.shape[3], t.shape[4],
-                  t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+    with arbitrary strides is fine as long as head_dim is contiguous).  Structs are cached by
+    (dtype, shape, strides): a decode loop asks for the same one every step."""
+    key = (t.dtype, tuple(t.shape), t.stride())
+    lay = _layout_cache.get(key)
+    if lay is None:
+        if t.dim() != 5 or t.stride(4) != 1:
+            raise FreqKVError(ERR_UNSUPPORTED, "cache must be [batch, layers, kv_heads, capacity, head_dim] with contiguous head_dim")
+        lay = Layout(dtype_code(t.dtype), t.shape[0], t.shape[1], t.shape[2], t.shape[3], t.shape[4],
+                     t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+        if len(_layout_cache) > 256:
+            _layout_cache.clear()
+        _layout_cache[key] = lay
+    return lay
 
 
 def layout_contiguous(dtype: int, batch: int, layers: int, kv_heads: int, capacity: int, head_dim: int):

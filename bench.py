@@ -397,7 +397,9 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
                        "l2": "%d layers alternate, %.2f GB read per call" % (layers, bytes_per_call / 1e9)},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": "copy, of " + peaks["source"],
-                         "kernel": "attend_partial_kernel + attend_merge_kernel", "kernel_ms": kernel_ms, "traffic": None},
+                         "kernel": ("attend_mma_kernel" if G >= 2 else "attend_partial_kernel") + " + attend_merge_kernel",
+                         "kernel_ms": kernel_ms,
+                         "traffic": None},
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 

@@ -200,6 +200,10 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
  *   q, out  DEVICE pointers, dense [batch, kv_heads * q_heads_per_kv, head_dim] in the cache dtype;
  *           query head i uses KV head i / q_heads_per_kv (grouped-query attention); q is given
  *           before RoPE; out = softmax(scale * q_rot . K_rot^T) V, fp32 arithmetic, rounded once.
+ *           bf16 caches with q_heads_per_kv >= 2 take both products on the tensor cores (fp32
+ *           accumulation): rotated keys and scaled queries are rounded to fp16 for the scores,
+ *           the softmax weights to bf16 for the second product; keys and  scale * log2(e) * q
+ *           must then stay below 65504 in magnitude (larger values give infinities).
  *   scale   score scale; <= 0 selects 1/sqrt(head_dim).
  *   lens    HOST array of `batch` cache lengths, each in [1, capacity].
  * Nothing in the cache is written.  Errors: INVALID_ARG (null pointers, q == out, layer out of

@@ -873,7 +873,7 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
         }
         table = ctx->rope_table;
     }
-    const int32_t splits = attend_splits(l.batch, l.kv_heads, max_len, q_heads_per_kv, ctx->sm_count);
+    const int32_t splits = attend_splits(l.batch, l.kv_heads, max_len, q_heads_per_kv, l.dtype, ctx->sm_count);
     const size_t need = attend_partial_bytes(splits, l.batch, l.kv_heads * q_heads_per_kv);
     if (need > ctx->attend_partial_bytes) {
         if (ctx->attend_partial) {

@@ -8,7 +8,7 @@ constexpr int ATTEND_MAX_BATCH = 128;  // sequences per launch (lengths travel a
 
 bool attend_supported(int32_t head_dim, int32_t q_heads_per_kv);
 // Row splits per (sequence, kv head) so that the launch fills the device.
-int32_t attend_splits(int32_t batch, int32_t kv_heads, int32_t max_len, int32_t q_heads_per_kv, int sm_count);
+int32_t attend_splits(int32_t batch, int32_t kv_heads, int32_t max_len, int32_t q_heads_per_kv, int32_t dtype, int sm_count);
 size_t attend_partial_bytes(int32_t splits, int32_t batch, int32_t q_heads);
 // table[pos][c] = (cos, sin)(pos * base^(-2c/128)), pos < rows, c < 64.
 cudaError_t launch_rope_table(float2* table, int32_t rows, double base, cudaStream_t stream);

@@ -1,4 +1,5 @@
-"""Decode-time attention over the compressed cache -- TEST INFRASTRUCTURE, not part of the product.
+"""Attention over the compressed cache (decoding and chunk-wise prefilling) -- TEST INFRASTRUCTURE,
+not part of the product.
 
 Plain fp64 numpy statement of Section 3.4 (the attention of a newly incoming token over sink
 tokens, compressed tokens and recent tokens, the second attention equation of that section)
@@ -68,4 +69,25 @@ def attend_decode(q, k_cache, v_cache, length: int, rope_base: float, scale: flo
         w /= w.sum()
         for j in range(length):
             out[g] += w[j] * V[j]
+    return out
+
+
+def attend_prefill(q, k_cache, v_cache, length: int, rope_base: float, scale: float | None = None) -> np.ndarray:
+    """Outputs of the attention of a chunk of incoming tokens (Section 3.3, chunk-wise processing
+    during training and prefilling, first attention equation).
+
+    The chunk's ``n`` tokens have been appended to the cache: they sit in rows
+    ``[length - n, length)``.  Token i of the chunk attends to the sink rows, the compressed rows,
+    the chunk's earlier tokens and itself, i.e. to cache rows ``[0, length - n + i]``; positions
+    are the row indices in the cache for keys and query alike.  That is the decoding step of the
+    cache as it stood when token i had just been appended, so that is how it is computed.
+    ``q``: ``[G, n, d]`` (before RoPE); returns ``[G, n, d]`` in fp64.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    G, n, d = q.shape
+    if not 1 <= n <= length:
+        raise ValueError("need 1 <= chunk length <= cache length")
+    out = np.empty((G, n, d))
+    for i in range(n):
+        out[:, i, :] = attend_decode(q[:, i, :], k_cache, v_cache, length - n + i + 1, rope_base, scale)
     return out

@@ -103,3 +103,55 @@ def test_output_is_a_convex_combination_of_the_value_rows():
     V = r.standard_normal((50, 12))
     out = oa.attend_decode(r.standard_normal((3, 12)) * 3, r.standard_normal((50, 12)), V, 50, 10000.0)
     assert np.all(out <= V.max(axis=0) + 1e-12) and np.all(out >= V.min(axis=0) - 1e-12)
+
+
+# ---- chunk-wise prefilling (Section 3.3): every token of a chunk, causally ----
+
+def test_prefill_of_one_token_is_the_decoding_step():
+    r = rng(31)
+    K, V, q = r.standard_normal((40, 16)), r.standard_normal((40, 16)), r.standard_normal((2, 1, 16))
+    assert np.array_equal(oa.attend_prefill(q, K, V, 33, 10000.0), oa.attend_decode(q[:, 0], K, V, 33, 10000.0)[:, None, :])
+
+
+def test_prefill_is_causal_and_ignores_rows_past_the_length():
+    r = rng(32)
+    K, V, q = r.standard_normal((30, 8)), r.standard_normal((30, 8)), r.standard_normal((1, 5, 8))
+    base = oa.attend_prefill(q, K, V, 20, 10000.0)
+    K2, V2 = K.copy(), V.copy()
+    K2[18:], V2[18:] = 7.0, -3.0           # rows of chunk tokens 3, 4 and everything after the cache length
+    got = oa.attend_prefill(q, K2, V2, 20, 10000.0)
+    assert np.array_equal(got[:, :3], base[:, :3])   # tokens 0..2 see rows 0..17 only
+    assert not np.allclose(got[:, 3:], base[:, 3:])
+
+
+def test_prefill_first_token_of_an_empty_history_returns_its_own_value():
+    r = rng(33)
+    K, V, q = r.standard_normal((6, 4)), r.standard_normal((6, 4)), r.standard_normal((3, 6, 4))
+    out = oa.attend_prefill(q, K, V, 6, 10000.0)      # the chunk is the whole cache: token 0 sees row 0 only
+    assert np.allclose(out[:, 0], np.broadcast_to(V[0], (3, 4)), atol=TOL)
+
+
+def test_prefill_matches_masked_matrix_softmax_without_rope():
+    # no RoPE: the textbook causal attention softmax(mask(Q K^T / sqrt d)) V with the chunk at the end
+    r = rng(34)
+    n, length, d = 7, 19, 8
+    K, V, q = r.standard_normal((25, d)), r.standard_normal((25, d)), r.standard_normal((2, n, d))
+    scores = torch.from_numpy(q) @ torch.from_numpy(K[:length]).T / math.sqrt(d)
+    rows = torch.arange(length)[None, :] <= (length - n + torch.arange(n))[:, None]
+    want = torch.softmax(scores.masked_fill(~rows, float("-inf")), dim=-1) @ torch.from_numpy(V[:length])
+    assert np.allclose(oa.attend_prefill(q, K, V, length, 0.0), want.numpy(), atol=TOL)
+
+
+def test_prefill_with_rope_matches_matrix_form():
+    # RoPE at in-cache positions written as matrices: rotate every key row by its index, every query by its row index
+    r = rng(35)
+    n, length, d, base = 4, 11, 16, 10000.0
+    K, V, q = r.standard_normal((12, d)), r.standard_normal((12, d)), r.standard_normal((1, n, d))
+    Kr = np.stack([oa.rope(K[j], j, base) for j in range(length)])
+    Qr = np.stack([oa.rope(q[0, i], length - n + i, base) for i in range(n)])
+    S = Qr @ Kr.T / math.sqrt(d)
+    for i in range(n):
+        S[i, length - n + i + 1:] = -np.inf
+    W = np.exp(S - S.max(axis=1, keepdims=True))
+    W /= W.sum(axis=1, keepdims=True)
+    assert np.allclose(oa.attend_prefill(q, K, V, length, base)[0], W @ V[:length], atol=TOL)

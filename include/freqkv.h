@@ -214,6 +214,28 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
                                    int32_t layer, const void* q, void* out, int32_t q_heads_per_kv, const int32_t* lens,
                                    float rope_base, float scale, void* cuda_stream);
 
+/* Attention of a chunk of n_new incoming tokens per sequence over the bounded cache of one layer
+ * (Section 3.3: during training and prefilling the sequence is processed chunk-wise, attention
+ * interleaved with compression; first attention equation).  The chunk's keys and values have been
+ * appended already: they are cache rows [lens[b] - n_new, lens[b]).  Token i of the chunk attends
+ * to the sink tokens, the compressed tokens, the chunk's earlier tokens and itself, i.e. to rows
+ * [0, lens[b] - n_new + i]; keys and queries get the RoPE of Section 3.4 at those row indices
+ * (key row j at j, query i at lens[b] - n_new + i; same pairing and rope_base rule as above).
+ *   q, out  DEVICE pointers, dense [batch, kv_heads * q_heads_per_kv, n_new, head_dim], bf16;
+ *           out = softmax(mask(scale * q_rot . K_rot^T)) V.  Both products run on the tensor
+ *           cores with fp32 accumulation: rotated keys and scaled queries are rounded to fp16,
+ *           the softmax weights to bf16; keys and  scale * log2(e) * q  must stay below 65504.
+ *   lens    HOST array of `batch` cache lengths (chunk included), each in [n_new, capacity].
+ * Nothing in the cache is written.  Errors: INVALID_ARG (null pointers, q == out, layer out of
+ * range, n_new < 1, a length outside [n_new, capacity], NaN scale or base), UNSUPPORTED (fp32
+ * caches, head_dim != 128, misaligned pointers, layout rules), ALLOC, CUDA.  The context keeps
+ * two scratch buffers (rotated keys of one layer, rotated queries of one chunk) and the cos/sin
+ * table.  A barrier wait inside the kernel that runs out (2 s) ends the kernel and shows up in
+ * freqkv_last_device_status as TIMEOUT. */
+freqkv_status freqkv_attend_prefill(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v,
+                                    int32_t layer, const void* q, void* out, int32_t q_heads_per_kv, int32_t n_new,
+                                    const int32_t* lens, float rope_base, float scale, void* cuda_stream);
+
 /* Instrumentation for benchmarks.  With timing enabled every compression records a CUDA event
  * pair on the caller's stream around its transform kernel (the projection / fast-transform
  * launch, not the copy-back or table builders).  freqkv_get_timing waits for the recorded
@@ -262,8 +284,8 @@ freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, void* k, void
 freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream);
 
 /* Host-only argument checks, exactly the ones freqkv_compress / freqkv_append apply before
- * they enqueue anything (they touch no device and need no context; freqkv_check_attend likewise
- * for freqkv_attend_decode): the status those calls
+ * they enqueue anything (they touch no device and need no context; freqkv_check_attend and
+ * freqkv_check_attend_prefill likewise for the two attention calls): the status those calls
  * would return for these arguments, FREQKV_OK if they would go ahead. */
 freqkv_status freqkv_check_compress(const freqkv_layout* layout, const void* k, const void* v, int32_t cache_len,
                                     int32_t kept_len, int32_t sink);
@@ -271,6 +293,9 @@ freqkv_status freqkv_check_append(const freqkv_layout* layout, const void* k, co
                                   const void* new_v, int32_t n_new, const int32_t* lens);
 freqkv_status freqkv_check_attend(const freqkv_layout* layout, const void* k, const void* v, int32_t layer, const void* q,
                                   const void* out, int32_t q_heads_per_kv, const int32_t* lens);
+freqkv_status freqkv_check_attend_prefill(const freqkv_layout* layout, const void* k, const void* v, int32_t layer,
+                                          const void* q, const void* out, int32_t q_heads_per_kv, int32_t n_new,
+                                          const int32_t* lens);
 
 /* Text of the most recent CUDA failure or device-status report seen by this context (owned by
  * the context, valid until its next call); "" if none. */

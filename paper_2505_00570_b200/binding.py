@@ -28,6 +28,7 @@ EXPORTS = [
     "freqkv_last_error", "freqkv_status_string", "freqkv_version", "freqkv_compress_host",
     "freqkv_set_timing", "freqkv_get_timing", "freqkv_compress_noalloc", "freqkv_attend_decode",
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
+    "freqkv_attend_prefill", "freqkv_check_attend_prefill",
     "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
@@ -89,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.freqkv_attend_decode.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, I32P,
                                            ctypes.c_float, ctypes.c_float, c_void_p]
         L.freqkv_check_attend.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, I32P]
+        L.freqkv_attend_prefill.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32,
+                                            I32P, ctypes.c_float, ctypes.c_float, c_void_p]
+        L.freqkv_check_attend_prefill.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, I32P]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -149,6 +153,12 @@ def check_append(layout: Layout, k_ptr: int, v_ptr: int, nk_ptr: int, nv_ptr: in
 def check_attend(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_ptr: int, out_ptr: int, group: int, lens) -> int:
     arr = (c_int32 * len(lens))(*lens)
     return lib().freqkv_check_attend(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, arr)
+
+
+def check_attend_prefill(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_ptr: int, out_ptr: int, group: int,
+                         n_new: int, lens) -> int:
+    arr = (c_int32 * len(lens))(*lens)
+    return lib().freqkv_check_attend_prefill(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, n_new, arr)
 
 
 def _stream_ptr(stream) -> int:
@@ -341,6 +351,27 @@ class Context:
                                         out.data_ptr(), q.shape[1] // lay.kv_heads, c_lens, rope_base, scale,
                                         _stream_ptr(stream))
         self._check(st, "freqkv_attend_decode")
+        return out
+
+    def attend_prefill(self, k: torch.Tensor, v: torch.Tensor, layer: int, q: torch.Tensor, lens: list[int],
+                       rope_base: float = 10000.0, scale: float = 0.0, out: torch.Tensor | None = None,
+                       stream=None) -> torch.Tensor:
+        """Causal attention of a chunk of tokens, already appended as cache rows [lens[b] - n_new, lens[b])
+        of `layer`, over rows [0, lens[b]) (keys and queries rotated to their in-cache positions).
+        ``q``: dense [batch, q_heads, n_new, head_dim], bf16, before RoPE.  Returns ``out``."""
+        lay = layout_of(k)
+        if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
+            raise FreqKVError(ERR_INVALID_ARG, "K and V must share shape, strides and dtype")
+        if q.dim() != 4 or not q.is_contiguous() or q.dtype != k.dtype or q.shape[0] != lay.batch or \
+                q.shape[3] != lay.head_dim or q.shape[1] % lay.kv_heads != 0:
+            raise FreqKVError(ERR_INVALID_ARG, "q must be dense [batch, q_heads, n_new, head_dim] in the cache dtype")
+        if out is None:
+            out = torch.empty_like(q)
+        c_lens = (c_int32 * lay.batch)(*lens)
+        st = lib().freqkv_attend_prefill(self._h, ctypes.byref(lay), k.data_ptr(), v.data_ptr(), layer, q.data_ptr(),
+                                         out.data_ptr(), q.shape[1] // lay.kv_heads, q.shape[2], c_lens, rope_base, scale,
+                                         _stream_ptr(stream))
+        self._check(st, "freqkv_attend_prefill")
         return out
 
     def compress_host(self, k_host: torch.Tensor, v_host: torch.Tensor, cache_len: int, kept_len: int, sink: int,

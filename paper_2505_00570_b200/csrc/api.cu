@@ -17,6 +17,7 @@
 #include "gemm.cuh"
 #include "fdct.cuh"
 #include "attend.cuh"
+#include "prefill.cuh"
 
 using namespace freqkv;
 
@@ -50,6 +51,10 @@ struct freqkv_ctx {
     double rope_base = 0.0;
     float* attend_partial = nullptr;
     size_t attend_partial_bytes = 0;
+    void* prefill_keys = nullptr;     // rotated keys of one layer, fp16
+    size_t prefill_keys_bytes = 0;
+    void* prefill_queries = nullptr;  // rotated, scaled queries of one chunk, fp16
+    size_t prefill_queries_bytes = 0;
     cudaStream_t pipe[3] = {nullptr, nullptr, nullptr};  // copy in, compress, copy out
     cudaEvent_t pipe_begin = nullptr, pipe_end = nullptr;
     std::vector<cudaEvent_t> pipe_events;                // per group: copied in, compressed
@@ -501,6 +506,8 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     if (ctx->work_done) cudaEventDestroy(ctx->work_done);
     if (ctx->rope_table) cudaFree(ctx->rope_table);
     if (ctx->attend_partial) cudaFree(ctx->attend_partial);
+    if (ctx->prefill_keys) cudaFree(ctx->prefill_keys);
+    if (ctx->prefill_queries) cudaFree(ctx->prefill_queries);
     for (int i = 0; i < 3; ++i)
         if (ctx->pipe[i]) cudaStreamDestroy(ctx->pipe[i]);
     if (ctx->pipe_begin) cudaEventDestroy(ctx->pipe_begin);
@@ -822,6 +829,30 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
     return FREQKV_OK;
 }
 
+// The context's cos/sin table for `rope_base`, built on `stream` when the base or the capacity has
+// changed; *table stays null when RoPE is off.
+static freqkv_status rope_table_for(freqkv_ctx* ctx, int32_t capacity, float rope_base, cudaStream_t stream, const float2** table)
+{
+    *table = nullptr;
+    if (!(rope_base > 0.f)) return FREQKV_OK;
+    if (!ctx->rope_table || ctx->rope_rows < capacity || ctx->rope_base != (double)rope_base) {
+        if (ctx->rope_table) {
+            FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // an enqueued launch may still read the old table
+            cudaFree(ctx->rope_table);
+            ctx->rope_table = nullptr;
+        }
+        const int32_t rows = std::max(capacity, 2);
+        FREQKV_CUDA(ctx, cudaMalloc(&ctx->rope_table, (size_t)rows * 64 * sizeof(float2)));
+        const cudaError_t e = launch_rope_table(ctx->rope_table, rows, (double)rope_base, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "rope_table");
+        ctx->rope_rows = rows;
+        ctx->rope_base = (double)rope_base;
+        ctx->kernels_launched += 1;
+    }
+    *table = ctx->rope_table;
+    return FREQKV_OK;
+}
+
 freqkv_status freqkv_check_attend(const freqkv_layout* layout, const void* k, const void* v, int32_t layer, const void* q,
                                   const void* out, int32_t q_heads_per_kv, const int32_t* lens)
 {
@@ -856,23 +887,8 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
     int32_t max_len = 0;
     for (int32_t b = 0; b < l.batch; ++b) max_len = std::max(max_len, lens[b]);
     const float2* table = nullptr;
-    if (rope_base > 0.f) {
-        if (!ctx->rope_table || ctx->rope_rows < l.capacity || ctx->rope_base != (double)rope_base) {
-            if (ctx->rope_table) {
-                FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // an enqueued launch may still read the old table
-                cudaFree(ctx->rope_table);
-                ctx->rope_table = nullptr;
-            }
-            const int32_t rows = std::max(l.capacity, 2);
-            FREQKV_CUDA(ctx, cudaMalloc(&ctx->rope_table, (size_t)rows * 64 * sizeof(float2)));
-            const cudaError_t e = launch_rope_table(ctx->rope_table, rows, (double)rope_base, stream);
-            if (e != cudaSuccess) return cuda_fail(ctx, e, "rope_table");
-            ctx->rope_rows = rows;
-            ctx->rope_base = (double)rope_base;
-            ctx->kernels_launched += 1;
-        }
-        table = ctx->rope_table;
-    }
+    const freqkv_status ts = rope_table_for(ctx, l.capacity, rope_base, stream, &table);
+    if (ts != FREQKV_OK) return ts;
     const int32_t splits = attend_splits(l.batch, l.kv_heads, max_len, q_heads_per_kv, l.dtype, ctx->sm_count);
     const size_t need = attend_partial_bytes(splits, l.batch, l.kv_heads * q_heads_per_kv);
     if (need > ctx->attend_partial_bytes) {
@@ -892,6 +908,80 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "attend");
     ctx->kernels_launched += 1 + (l.batch + ATTEND_MAX_BATCH - 1) / ATTEND_MAX_BATCH;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_check_attend_prefill(const freqkv_layout* layout, const void* k, const void* v, int32_t layer,
+                                          const void* q, const void* out, int32_t q_heads_per_kv, int32_t n_new,
+                                          const int32_t* lens)
+{
+    if (!lens) return FREQKV_ERR_INVALID_ARG;
+    freqkv_status st = check_layout(layout);
+    if (st != FREQKV_OK) return st;
+    st = check_tensors(*layout, k, v);
+    if (st != FREQKV_OK) return st;
+    if (!q || !out || q == out) return FREQKV_ERR_INVALID_ARG;
+    if (((uintptr_t)q | (uintptr_t)out) & 15) return FREQKV_ERR_UNSUPPORTED;
+    if (layer < 0 || layer >= layout->layers || q_heads_per_kv < 1 || n_new < 1) return FREQKV_ERR_INVALID_ARG;
+    if (!prefill_supported(layout->dtype, layout->head_dim, q_heads_per_kv)) return FREQKV_ERR_UNSUPPORTED;
+    for (int32_t b = 0; b < layout->batch; ++b)
+        if (lens[b] < n_new || lens[b] > layout->capacity) return FREQKV_ERR_INVALID_ARG;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_attend_prefill(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v, int32_t layer,
+                                    const void* q, void* out, int32_t q_heads_per_kv, int32_t n_new, const int32_t* lens,
+                                    float rope_base, float scale, void* cuda_stream)
+{
+    if (!ctx) return FREQKV_ERR_INVALID_ARG;
+    const freqkv_status st = freqkv_check_attend_prefill(layout, k, v, layer, q, out, q_heads_per_kv, n_new, lens);
+    if (st != FREQKV_OK) return st;
+    if (!(scale == scale) || !(rope_base == rope_base)) return FREQKV_ERR_INVALID_ARG;  // NaN
+    const freqkv_layout& l = *layout;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    WorkOrder order(ctx, stream);
+    if (scale <= 0.f) scale = 1.0f / sqrtf((float)l.head_dim);
+    const float2* table = nullptr;
+    const freqkv_status ts = rope_table_for(ctx, l.capacity, rope_base, stream, &table);
+    if (ts != FREQKV_OK) return ts;
+    struct Grow { void** p; size_t* have; size_t need; };
+    const Grow scratch[2] = {{&ctx->prefill_keys, &ctx->prefill_keys_bytes, prefill_key_scratch_bytes(l)},
+                             {&ctx->prefill_queries, &ctx->prefill_queries_bytes, prefill_query_scratch_bytes(l, q_heads_per_kv, n_new)}};
+    for (const Grow& s : scratch) {
+        if (s.need <= *s.have) continue;
+        if (*s.p) {
+            FREQKV_CUDA(ctx, cudaDeviceSynchronize());  // an enqueued launch may still use the old buffer
+            cudaFree(*s.p);
+            *s.p = nullptr;
+            *s.have = 0;
+        }
+        if (cudaMalloc(s.p, s.need) != cudaSuccess) {
+            cudaGetLastError();
+            *s.p = nullptr;
+            ctx->last_error = "out of device memory for the prefill attention scratch";
+            return FREQKV_ERR_ALLOC;
+        }
+        *s.have = s.need;
+    }
+    const char* why = nullptr;
+    int32_t launched = 0;
+    cudaError_t e;
+    {
+        TransformTimer timer(ctx, stream);
+        e = launch_prefill(l, k, v, layer, q, out, q_heads_per_kv, n_new, lens, table, scale, ctx->prefill_keys,
+                           ctx->prefill_queries, ctx->status_dev, &why, &launched, stream);
+    }
+    ctx->kernels_launched += launched;
+    if (e != cudaSuccess) {
+        if (why) {
+            cudaGetLastError();
+            ctx->last_error = why;
+            return e == cudaErrorNotSupported ? FREQKV_ERR_UNSUPPORTED : FREQKV_ERR_CUDA;
+        }
+        return cuda_fail(ctx, e, "attend_prefill");
+    }
     return FREQKV_OK;
 }
 

@@ -141,6 +141,23 @@ def test_check_attend():
     assert fk.check_attend(lay(hd=64), K, V, 0, Q, O, 1, [10]) == fk.ERR_UNSUPPORTED
 
 
+def test_check_attend_prefill():
+    L = lay(cap=64, B=2)
+    Q, O = 0x30000000, 0x40000000
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 1, 10, [10, 64]) == fk.OK
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 3, 1, [1, 20]) == fk.OK                 # any group size
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 1, 0, [10, 20]) == fk.ERR_INVALID_ARG   # an empty chunk
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 1, 11, [10, 20]) == fk.ERR_INVALID_ARG  # chunk longer than a cache length
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 1, 5, [10, 65]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend_prefill(L, K, V, 0, Q, O, 0, 5, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend_prefill(L, K, V, L.layers, Q, O, 1, 5, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend_prefill(L, K, V, 0, Q, Q, 1, 5, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend_prefill(L, K, V, 0, 0, O, 1, 5, [10, 20]) == fk.ERR_INVALID_ARG
+    assert fk.check_attend_prefill(L, K, V, 0, Q + 2, O, 1, 5, [10, 20]) == fk.ERR_UNSUPPORTED
+    assert fk.check_attend_prefill(lay(hd=64), K, V, 0, Q, O, 1, 5, [10]) == fk.ERR_UNSUPPORTED
+    assert fk.check_attend_prefill(lay(dtype=fk.F32), K, V, 0, Q, O, 1, 5, [10]) == fk.ERR_UNSUPPORTED  # bf16 caches only
+
+
 def test_null_context_is_rejected():
     L = lay()
     lib = fk.lib()

@@ -403,6 +403,52 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 
+def run_prefill_attend(args, ctx, fk, synth, dev, peaks):
+    """Chunk-wise prefilling attention (Section 3.3) of one 7B-shaped layer: the 2046 tokens that
+    refill the cache after a compression attend causally to 4 sinks + 2046 compressed rows + the
+    chunk.  One freqkv_attend_prefill call per step, layers alternating."""
+    B, H, G, cap, base = 1, 32, 1, 4096, 10000.0
+    n_new = cap - 4 - (cap - 4) // 2
+    layers = 4
+    w = synth.Workload("prefill_attend_7b", B, layers, H, 128, cap, torch.bfloat16, 4, 0.9, 2, synth.BASE_SEED + 8)
+    k, v = synth.make_cache(w, dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed + 1)
+    q = torch.randn(B, H * G, n_new, 128, generator=gen, device=dev).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    lens = [cap] * B
+    pos0 = cap - n_new
+    attended = n_new * pos0 + n_new * (n_new + 1) // 2          # (query, key) pairs under the causal mask, per head
+    flops_per_call = 4 * 128 * attended * B * H * G             # two products, 2 flop per multiply-add
+    for i in range(max(args.warmup, 3)):
+        ctx.attend_prefill(k, v, i % layers, q, lens, rope_base=base, out=out)
+    torch.cuda.synchronize()
+    ctx.get_timing()
+    ctx.set_timing(True)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(args.steps):
+        ctx.attend_prefill(k, v, i % layers, q, lens, rope_base=base, out=out)
+    b.record()
+    torch.cuda.synchronize()
+    n, t_ms, _ = ctx.get_timing()
+    ctx.set_timing(False)
+    ms = a.elapsed_time(b) / args.steps
+    kernel_ms = t_ms / max(n, 1)
+    achieved = flops_per_call / (kernel_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    return {"metric": "prefill attention TFLOP/s (causal pairs only)", "value": flops_per_call / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "prefill_attend_7b", "batch": B, "kv_heads": H, "q_heads_per_kv": G, "head_dim": 128,
+                       "cache_len": cap, "chunk": n_new, "rope_base": base,
+                       "step": "one freqkv_attend_prefill call over one layer", "l2": "%d layers alternate" % layers},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_kind": "cuBLAS bf16 burst, of " + peaks["source"],
+                         "kernel": "prefill_rope_kernel + prefill_attend_kernel", "kernel_ms": kernel_ms, "traffic": None},
+            "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
+
+
 def run_spectrum(args, ctx, fk, synth, dev, peaks):
     """Average DCT power spectrum of a 7B-shaped cache (Section 3.1): one freqkv_power_spectrum call per step."""
     w = synth.WORKLOADS["llama2_7b"]
@@ -474,6 +520,15 @@ def main():
             torch.cuda.set_device(local_rank)
             ctx = fk.Context(local_rank)
             print(json.dumps(run_spectrum(args, ctx, fk, synth, torch.device("cuda", local_rank), load_peaks())), flush=True)
+            ctx.close()
+        return
+    if args.workload == "prefill_attend_7b":          # side workload: chunk-wise prefilling attention
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            ctx = fk.Context(local_rank)
+            print(json.dumps(run_prefill_attend(args, ctx, fk, synth, torch.device("cuda", local_rank), load_peaks())), flush=True)
             ctx.close()
         return
     if args.workload in ("attend_7b", "attend_8b"):   # side workload: the step after the compression path

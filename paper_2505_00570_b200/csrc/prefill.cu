@@ -13,8 +13,10 @@
 //     them to fp16 into scratch (fp16 rather than bf16: three more mantissa bits keep the error of
 //     the scores a quarter of bf16's).  Key rows from the length to the next multiple of 128 are
 //     written as zeros.
-//   pass 2, one CTA per (sequence, query head, 128 queries), 192 threads:
-//     warp 0   TMA producer: the query tile once; per key tile of 128 rows the rotated keys and,
+//   pass 2, one CTA per (sequence, query head, 128 queries), 192 threads, two CTAs per SM (each
+//   holds half of the shared memory and of the tensor memory, so that one CTA's softmax overlaps
+//   the other's tensor-core work); the query tiles with the most keys are scheduled first:
+//     warp 0   TMA producer: the query tile once; per key tile of 64 rows the rotated keys and,
 //              straight from the cache through a 5-D tensor map, the values (two-stage rings);
 //     warp 1   MMA issuer: S = Q K_rot^T (fp16 in, fp32 in tensor memory, two S buffers so that
 //              the next tile's scores are computed while this tile's softmax runs), then
@@ -41,20 +43,29 @@ namespace freqkv {
 namespace {
 
 constexpr int BQ = 128;             // queries per CTA
-constexpr int BKV = 128;            // keys per tile
-constexpr int SLAB = 128 * 128;     // bytes: 128 rows x 64 two-byte values, one 128-byte swizzle row each
-constexpr int TILE = 2 * SLAB;      // 128 rows x 128 values
+constexpr int BKV = 64;             // keys per tile
+constexpr int Q_SLAB = BQ * 128;    // bytes: 128 rows x 64 two-byte values, one 128-byte swizzle row each
+constexpr int Q_TILE = 2 * Q_SLAB;  // 128 queries x 128 channels
+constexpr int P_TILE = BQ * 128;    // 128 queries x 64 keys
+constexpr int KV_SLAB = BKV * 128;  // 64 rows x 64 channels
+constexpr int KV_TILE = 2 * KV_SLAB;
 constexpr int RING = 2;             // stages of the key ring and of the value ring
-constexpr int OFF_Q = 0, OFF_P = TILE, OFF_K = 2 * TILE, OFF_V = OFF_K + RING * TILE, OFF_BAR = OFF_V + RING * TILE;
-constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024 /* alignment slack */;
+constexpr int OFF_Q = 0, OFF_P = Q_TILE, OFF_K = OFF_P + P_TILE, OFF_V = OFF_K + RING * KV_TILE, OFF_BAR = OFF_V + RING * KV_TILE;
+constexpr int SMEM_USED = OFF_BAR + 256;
+// Two CTAs share an SM's 228 KB (1 KB of each CTA's share is reserved): 115712 bytes each at most.
+// The tiles need a 1024-byte aligned base; the slack left for aligning it is 768 bytes, and the
+// kernel checks that it was enough (a base that is 1024-aligned already needs none).
+constexpr int SMEM_BYTES = 115712;
+static_assert(SMEM_USED <= SMEM_BYTES, "the tiles of a CTA must leave room for a second CTA on the SM");
 constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 256;      // S buffers in columns 0..63 and 64..127, O in 128..255
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 constexpr unsigned long long LANDING_NS = 1000000ull;        // 1 ms
 constexpr float NEG_INF = -INFINITY;
 constexpr float RESCALE_STEP = 8.f;  // log2 of the largest weight the lazy reference allows
 
 struct PrefillParams {
-    int32_t n_new, kv_heads, g, layer, batch0;
+    int32_t n_new, kv_heads, g, layer, batch0, batch_count, q_tiles;
     __nv_bfloat16* out;  // [batch, kv_heads * g, n_new, 128]
     int32_t* status;
     int32_t len[PREFILL_MAX_BATCH];
@@ -142,9 +153,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;
     return d;
 }
-// Instruction descriptors, kind::f16, D fp32, M = 128, N = 128.
-// Scores: A and B fp16, both K-major.  Values: A and B bf16, A K-major, B MN-major.
-constexpr uint32_t IDESC_QK = (1u << 4) | (0u << 7) | (0u << 10) | (0u << 15) | (0u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptors, kind::f16, D fp32, M = 128.
+// Scores (N = 64 keys): A and B fp16, both K-major.  Values (N = 128 channels): A and B bf16, A K-major, B MN-major.
+constexpr uint32_t IDESC_QK = (1u << 4) | (0u << 7) | (0u << 10) | (0u << 15) | (0u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t IDESC_PV = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
@@ -220,64 +231,73 @@ struct RopeJob {
 
 __global__ void __launch_bounds__(256) prefill_rope_kernel(const RopeJob job)
 {
+    // blockIdx.y: a (sequence, kv head) slice of keys, then the (sequence, query head) slices of queries;
+    // blockIdx.x: 64 consecutive rows of the slice, 4 per half-warp
     const int l16 = threadIdx.x % 16, c0 = 4 * l16;
-    const int64_t k_jobs = (int64_t)job.batch_count * job.kv_heads * job.k_rows;
-    const int64_t q_jobs = (int64_t)job.batch_count * job.heads_q * job.n_new;
-    for (int64_t r = (int64_t)blockIdx.x * 16 + threadIdx.x / 16; r < k_jobs + q_jobs; r += (int64_t)gridDim.x * 16) {
-        const __nv_bfloat16* src;
-        __half* dst;
-        int32_t pos;
-        float mul = 1.f;
-        bool zero = false;
-        if (r < k_jobs) {
-            const int32_t row = (int32_t)(r % job.k_rows), bh = (int32_t)(r / job.k_rows), b = bh / job.kv_heads, h = bh % job.kv_heads;
-            src = job.k + (int64_t)(job.batch0 + b) * job.stride_batch + (int64_t)h * job.stride_head + (int64_t)row * job.stride_token;
-            dst = job.k_out + (((int64_t)(job.batch0 + b) * job.kv_heads + h) * job.capacity + row) * 128;
-            pos = row;
-            zero = row >= job.len[b];
-        } else {
-            const int64_t rq = r - k_jobs;
-            const int32_t i = (int32_t)(rq % job.n_new), bh = (int32_t)(rq / job.n_new), b = bh / job.heads_q;
-            const int64_t at = ((int64_t)(job.batch0 + b) * job.heads_q + bh % job.heads_q) * job.n_new + i;
-            src = job.q + at * 128;
-            dst = job.q_out + at * 128;
-            pos = job.len[b] - job.n_new + i;
-            mul = job.qscale;
-        }
+    const int32_t k_slices = job.batch_count * job.kv_heads;
+    const bool is_key = (int32_t)blockIdx.y < k_slices;
+    const int32_t slice = is_key ? (int32_t)blockIdx.y : (int32_t)blockIdx.y - k_slices;
+    const int32_t heads = is_key ? job.kv_heads : job.heads_q, b = slice / heads, hh = slice % heads;
+    const int32_t rows = is_key ? job.k_rows : job.n_new, len = job.len[b];
+    const __nv_bfloat16* src0;
+    __half* dst0;
+    int64_t src_stride;
+    if (is_key) {
+        src0 = job.k + (int64_t)(job.batch0 + b) * job.stride_batch + (int64_t)hh * job.stride_head;
+        src_stride = job.stride_token;
+        dst0 = job.k_out + ((int64_t)(job.batch0 + b) * job.kv_heads + hh) * job.capacity * 128;
+    } else {
+        const int64_t at = ((int64_t)(job.batch0 + b) * job.heads_q + hh) * job.n_new * 128;
+        src0 = job.q + at;
+        src_stride = 128;
+        dst0 = job.q_out + at;
+    }
+    const float mul = is_key ? 1.f : job.qscale;
+    const int32_t pos0 = is_key ? 0 : len - job.n_new;
+#pragma unroll
+    for (int i4 = 0; i4 < 4; ++i4) {
+        const int32_t row = (int32_t)blockIdx.x * 64 + (threadIdx.x / 16) * 4 + i4;
+        if (row >= rows) break;
         uint2 lo_out = make_uint2(0u, 0u), hi_out = make_uint2(0u, 0u);
-        if (!zero) {
+        if (!(is_key && row >= len)) {  // key rows from the length on are written as zeros
+            const __nv_bfloat16* src = src0 + (int64_t)row * src_stride;
             const uint2 ulo = __ldg(reinterpret_cast<const uint2*>(src + c0)), uhi = __ldg(reinterpret_cast<const uint2*>(src + 64 + c0));
             float lo[4] = {__uint_as_float(ulo.x << 16), __uint_as_float(ulo.x & 0xffff0000u), __uint_as_float(ulo.y << 16),
                            __uint_as_float(ulo.y & 0xffff0000u)};
             float hi[4] = {__uint_as_float(uhi.x << 16), __uint_as_float(uhi.x & 0xffff0000u), __uint_as_float(uhi.y << 16),
                            __uint_as_float(uhi.y & 0xffff0000u)};
+            if (job.table) {
+                const float4* t = reinterpret_cast<const float4*>(job.table + (int64_t)(pos0 + row) * 64 + c0);
+                const float4 t0 = __ldg(t), t1 = __ldg(t + 1);
+                const float cs[4] = {t0.x, t0.z, t1.x, t1.z}, sn[4] = {t0.y, t0.w, t1.y, t1.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                if (job.table) {
-                    const float2 cs = __ldg(job.table + (int64_t)pos * 64 + c0 + i);
-                    const float a = lo[i] * cs.x - hi[i] * cs.y, bb = hi[i] * cs.x + lo[i] * cs.y;
+                for (int i = 0; i < 4; ++i) {
+                    const float a = lo[i] * cs[i] - hi[i] * sn[i], bb = hi[i] * cs[i] + lo[i] * sn[i];
                     lo[i] = a;
                     hi[i] = bb;
                 }
-                lo[i] *= mul;
-                hi[i] *= mul;
             }
-            lo_out = make_uint2(pack_f16(lo[0], lo[1]), pack_f16(lo[2], lo[3]));
-            hi_out = make_uint2(pack_f16(hi[0], hi[1]), pack_f16(hi[2], hi[3]));
+            lo_out = make_uint2(pack_f16(lo[0] * mul, lo[1] * mul), pack_f16(lo[2] * mul, lo[3] * mul));
+            hi_out = make_uint2(pack_f16(hi[0] * mul, hi[1] * mul), pack_f16(hi[2] * mul, hi[3] * mul));
         }
+        __half* dst = dst0 + (int64_t)row * 128;
         *reinterpret_cast<uint2*>(dst + c0) = lo_out;
         *reinterpret_cast<uint2*>(dst + 64 + c0) = hi_out;
     }
 }
 
 // ---- pass 2 ----
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS, 2)
 prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v, const PrefillParams prm)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
+    if (base - raw + SMEM_USED > SMEM_BYTES) {     // uniform over the CTA; nothing has been set up yet
+        if (threadIdx.x == 0) atomicOr(prm.status, PREFILL_ERR_WAIT);
+        return;
+    }
     uint8_t* aligned = smem_raw + (base - raw);
     const uint32_t bar0 = base + OFF_BAR;
     // barriers: q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_free[2], p_ready, o_full
@@ -293,8 +313,10 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int32_t b = blockIdx.z, hq = blockIdx.y, h = hq / prm.g;
-    const int32_t q_tile = (int32_t)(gridDim.x - 1 - blockIdx.x);  // the tiles with the most keys first
+    // heaviest work first: the first blocks are the last query tiles (the most keys) of all heads
+    const int32_t heads_q = prm.kv_heads * prm.g, units = heads_q * prm.batch_count;
+    const int32_t q_tile = prm.q_tiles - 1 - (int32_t)blockIdx.x / units;
+    const int32_t unit = (int32_t)blockIdx.x % units, b = unit / heads_q, hq = unit % heads_q, h = hq / prm.g;
     const int32_t q0 = q_tile * BQ;
     const int32_t len = prm.len[b], pos0 = len - prm.n_new;         // position of the chunk's first token
     const int32_t last_pos = pos0 + min(q0 + BQ, prm.n_new) - 1;    // of this tile's last valid query
@@ -316,33 +338,34 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {  // tensor memory: S buffers in columns 0..127 and 128..255, O in 256..383
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 128;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const int32_t q_slice = (prm.batch0 + b) * prm.kv_heads * prm.g + hq, k_slice = (prm.batch0 + b) * prm.kv_heads + h;
-            mbar_expect_tx(q_full, TILE);
+            const int32_t q_slice = (prm.batch0 + b) * heads_q + hq, k_slice = (prm.batch0 + b) * prm.kv_heads + h;
+            mbar_expect_tx(q_full, Q_TILE);
             tma_load_3d(base + OFF_Q, &map_q, q_full, 0, q0, q_slice);
-            tma_load_3d(base + OFF_Q + SLAB, &map_q, q_full, 64, q0, q_slice);
+            tma_load_3d(base + OFF_Q + Q_SLAB, &map_q, q_full, 64, q0, q_slice);
             for (int32_t t = 0; t < n_tiles; ++t) {
                 const int s = t % RING;
                 const uint32_t use = (uint32_t)(t / RING);
                 if (t >= RING && !mbar_wait(k_empty(s), (use - 1) & 1, abort_flag, prm.status)) break;
-                mbar_expect_tx(k_full(s), TILE);
-                tma_load_3d(base + OFF_K + s * TILE, &map_k, k_full(s), 0, t * BKV, k_slice);
-                tma_load_3d(base + OFF_K + s * TILE + SLAB, &map_k, k_full(s), 64, t * BKV, k_slice);
+                mbar_expect_tx(k_full(s), KV_TILE);
+                tma_load_3d(base + OFF_K + s * KV_TILE, &map_k, k_full(s), 0, t * BKV, k_slice);
+                tma_load_3d(base + OFF_K + s * KV_TILE + KV_SLAB, &map_k, k_full(s), 64, t * BKV, k_slice);
                 if (t >= RING && !mbar_wait(v_empty(s), (use - 1) & 1, abort_flag, prm.status)) break;
-                mbar_expect_tx(v_full(s), TILE);
-                tma_load_5d(base + OFF_V + s * TILE, &map_v, v_full(s), 0, t * BKV, h, prm.layer, prm.batch0 + b);
-                tma_load_5d(base + OFF_V + s * TILE + SLAB, &map_v, v_full(s), 64, t * BKV, h, prm.layer, prm.batch0 + b);
+                mbar_expect_tx(v_full(s), KV_TILE);
+                tma_load_5d(base + OFF_V + s * KV_TILE, &map_v, v_full(s), 0, t * BKV, h, prm.layer, prm.batch0 + b);
+                tma_load_5d(base + OFF_V + s * KV_TILE + KV_SLAB, &map_v, v_full(s), 64, t * BKV, h, prm.layer, prm.batch0 + b);
             }
             if (*abort_flag) {  // let the copies in flight land before this CTA's shared memory goes away
                 const unsigned long long t0 = global_timer_ns();
@@ -357,14 +380,13 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 const int s = t % RING;
                 const uint32_t use = (uint32_t)(t / RING);
                 if (!mbar_wait(k_full(s), use & 1, abort_flag, prm.status)) return false;
-                if (t >= 2 && !mbar_wait(s_free(t & 1), (use - 1) & 1, abort_flag, prm.status)) return false;
+                if (t >= 2 && !mbar_wait(s_free(t & 1), ((uint32_t)(t / 2) - 1) & 1, abort_flag, prm.status)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t qa = base + OFF_Q, ka = base + OFF_K + s * TILE;
+                const uint32_t qa = base + OFF_Q, ka = base + OFF_K + s * KV_TILE;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {  // 16 channels per instruction; 64-channel slabs, 32 bytes per step inside one
-                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
-                    umma(tmem_base + (t & 1) * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK, kk != 0);
-                }
+                for (int kk = 0; kk < 8; ++kk)  // 16 channels per instruction; 64-channel slabs, 32 bytes per step inside one
+                    umma(tmem_base + (t & 1) * BKV, smem_desc(qa + (kk / 4) * Q_SLAB + (kk % 4) * 32, 16, 1024),
+                         smem_desc(ka + (kk / 4) * KV_SLAB + (kk % 4) * 32, 16, 1024), IDESC_QK, kk != 0);
                 umma_commit(s_full(t & 1));
                 umma_commit(k_empty(s));
                 return true;
@@ -376,14 +398,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 if (!mbar_wait(p_ready, t & 1, abort_flag, prm.status)) break;
                 if (!mbar_wait(v_full(s), (t / RING) & 1, abort_flag, prm.status)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t pa = base + OFF_P, va = base + OFF_V + s * TILE;
+                const uint32_t pa = base + OFF_P, va = base + OFF_V + s * KV_TILE;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {  // 16 keys per instruction
-                    // P: K-major, 64-key slabs.  V: MN-major, 16 key rows = 2 KB per step, 64-channel slabs one SLAB apart.
-                    const uint64_t ad = smem_desc(pa + (kk / 4) * SLAB + (kk % 4) * 32, 16, 1024);
-                    const uint64_t bd = smem_desc(va + kk * 2048, SLAB, 1024);
-                    umma(tmem_base + 256, ad, bd, IDESC_PV, (t | kk) != 0);
-                }
+                for (int kk = 0; kk < BKV / 16; ++kk)  // 16 keys per instruction
+                    // P: K-major, one 64-key slab.  V: MN-major, 16 key rows = 2 KB per step, 64-channel slabs KV_SLAB apart.
+                    umma(tmem_o, smem_desc(pa + kk * 32, 16, 1024), smem_desc(va + kk * 2048, KV_SLAB, 1024), IDESC_PV, (t | kk) != 0);
                 umma_commit(o_full);
                 umma_commit(v_empty(s));
             }
@@ -391,7 +410,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     } else {
         // ---------------- softmax and epilogue: one query row per thread ----------------
         const int quarter = warp % 4, row = quarter * 32 + lane;     // tensor-memory lane = row of the tile
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t lane_bits = (uint32_t)(quarter * 32) << 16;
         const int32_t my_pos = pos0 + q0 + row;                      // keys up to this index are visible
         const int32_t warp_pos = pos0 + q0 + quarter * 32;           // the smallest position in this warp
         uint8_t* p_row = aligned + OFF_P + row * 128;
@@ -399,27 +418,26 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         bool alive = true;
         for (int32_t t = 0; t < n_tiles; ++t) {
             const int buf = t & 1, s = t % RING;
+            const int32_t j0 = t * BKV;
             if (!mbar_wait(s_full(buf), (t / 2) & 1, abort_flag, prm.status)) { alive = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            uint32_t sc[128];
-            tmem_ld32<0>(lane_addr + buf * 128 + 0, sc);
-            tmem_ld32<32>(lane_addr + buf * 128 + 32, sc);
-            tmem_ld32<64>(lane_addr + buf * 128 + 64, sc);
-            tmem_ld32<96>(lane_addr + buf * 128 + 96, sc);
+            uint32_t sc[64];
+            tmem_ld32<0>(tmem_base + lane_bits + buf * BKV + 0, sc);
+            tmem_ld32<32>(tmem_base + lane_bits + buf * BKV + 32, sc);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(s_free(buf));
 
-            const int32_t j0 = t * BKV;
             if (j0 + BKV - 1 > warp_pos) {  // a tile on the diagonal: hide the keys after each row's own
 #pragma unroll
-                for (int j = 0; j < 128; ++j)
+                for (int j = 0; j < 64; ++j)
                     if (j0 + j > my_pos) sc[j] = __float_as_uint(NEG_INF);
             }
-            float mx = NEG_INF;
+            float m4[4] = {NEG_INF, NEG_INF, NEG_INF, NEG_INF};  // four chains instead of one of 64
 #pragma unroll
-            for (int j = 0; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(sc[j]));
+            for (int j = 0; j < 64; ++j) m4[j & 3] = fmaxf(m4[j & 3], __uint_as_float(sc[j]));
+            const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
             // move the reference only when the maximum has outgrown it by more than RESCALE_STEP
             float factor = 1.f;
             const bool grow = mx > m_ref + RESCALE_STEP;   // true at the first tile (m_ref = -inf, key 0 is visible to every row)
@@ -428,15 +446,15 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 l_run *= factor;
                 m_ref = mx;
             }
-            uint32_t pk[64];
-            float sum = 0.f;
+            uint32_t pk[32];
+            float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int j = 0; j < 64; ++j) {
+            for (int j = 0; j < 32; ++j) {
                 const float p0 = ex2(__uint_as_float(sc[2 * j]) - m_ref), p1 = ex2(__uint_as_float(sc[2 * j + 1]) - m_ref);
-                sum += p0 + p1;
+                s4[j & 3] += p0 + p1;
                 pk[j] = pack_bf16(p0, p1);
             }
-            l_run += sum;
+            l_run += (s4[0] + s4[1]) + (s4[2] + s4[3]);
 
             if (t > 0) {  // the previous tile's P V must have finished: P is free, O is at rest
                 if (!mbar_wait(o_full, (t - 1) & 1, abort_flag, prm.status)) { alive = false; break; }
@@ -445,31 +463,28 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t o[32];
-                        tmem_ld32<0>(lane_addr + 256 + c * 32, o);
+                        tmem_ld32<0>(tmem_o + lane_bits + c * 32, o);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                         for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
-                        tmem_st32(lane_addr + 256 + c * 32, o);
+                        tmem_st32(tmem_o + lane_bits + c * 32, o);
                     }
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             }
-            // weights into shared memory: K-major operand, 64-key slabs, 16-byte chunks XOR-swizzled by the row
+            // weights into shared memory: K-major operand, 16-byte chunks XOR-swizzled by the row
 #pragma unroll
-            for (int slab = 0; slab < 2; ++slab)
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(p_row + slab * SLAB + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(pk[slab * 32 + c * 4], pk[slab * 32 + c * 4 + 1], pk[slab * 32 + c * 4 + 2], pk[slab * 32 + c * 4 + 3]);
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
             if (j0 + BKV > len) {  // value rows past the cache length are stale: make them zeros
                 if (!mbar_wait(v_full(s), (t / RING) & 1, abort_flag, prm.status)) { alive = false; break; }
-                if (j0 + row >= len) {
-                    uint8_t* v_row = aligned + OFF_V + s * TILE + row * 128;
+                if (row < BKV && j0 + row >= len) {
+                    uint8_t* v_row = aligned + OFF_V + s * KV_TILE + row * 128;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         *reinterpret_cast<uint4*>(v_row + c * 16) = make_uint4(0u, 0u, 0u, 0u);
-                        *reinterpret_cast<uint4*>(v_row + SLAB + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4*>(v_row + KV_SLAB + c * 16) = make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
             }
@@ -480,12 +495,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const float inv = 1.f / l_run;
             const bool store = q0 + row < prm.n_new;
-            uint4* out = reinterpret_cast<uint4*>(
-                prm.out + ((((int64_t)(prm.batch0 + b) * prm.kv_heads * prm.g + hq) * prm.n_new + q0 + row) * 128));
+            uint4* out = reinterpret_cast<uint4*>(prm.out + ((((int64_t)(prm.batch0 + b) * heads_q + hq) * prm.n_new + q0 + row) * 128));
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
-                tmem_ld32<0>(lane_addr + 256 + c * 32, o);
+                tmem_ld32<0>(tmem_o + lane_bits + c * 32, o);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (store) {
 #pragma unroll
@@ -503,7 +517,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS));
     }
 }
 
@@ -527,12 +541,12 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// fp16 scratch as (channel, row, slice); rows past the extent read as zeros.
-bool encode_rows_map(CUtensorMap* map, void* base, int64_t rows, int64_t slices)
+// fp16 scratch as (channel, row, slice), read in boxes of 64 channels x box_rows rows; rows past the extent read as zeros.
+bool encode_rows_map(CUtensorMap* map, void* base, int64_t rows, int64_t slices, uint32_t box_rows)
 {
     const cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)slices};
     const cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
-    const cuuint32_t box[3] = {64, 128, 1};
+    const cuuint32_t box[3] = {64, box_rows, 1};
     const cuuint32_t elem[3] = {1, 1, 1};
     return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -547,7 +561,7 @@ bool encode_value_map(CUtensorMap* map, const freqkv_layout& l, const void* v)
     const cuuint64_t strides[4] = {row, l.kv_heads > 1 ? (cuuint64_t)l.stride_head * 2 : row,
                                    l.layers > 1 ? (cuuint64_t)l.stride_layer * 2 : row,
                                    l.batch > 1 ? (cuuint64_t)l.stride_batch * 2 : row};
-    const cuuint32_t box[5] = {64, 128, 1, 1, 1};
+    const cuuint32_t box[5] = {64, BKV, 1, 1, 1};
     const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
     return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(v), dims, strides, box, elem,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -580,14 +594,16 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
     }
     static bool attr_set = false;
     if (!attr_set) {
-        const cudaError_t e = cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     const int32_t heads_q = l.kv_heads * g;
     CUtensorMap map_q, map_k, map_v;
-    if (!encode_rows_map(&map_q, query_scratch, n_new, (int64_t)l.batch * heads_q) ||
-        !encode_rows_map(&map_k, key_scratch, l.capacity, (int64_t)l.batch * l.kv_heads) || !encode_value_map(&map_v, l, v)) {
+    if (!encode_rows_map(&map_q, query_scratch, n_new, (int64_t)l.batch * heads_q, BQ) ||
+        !encode_rows_map(&map_k, key_scratch, l.capacity, (int64_t)l.batch * l.kv_heads, BKV) || !encode_value_map(&map_v, l, v)) {
         *error = "cuTensorMapEncodeTiled rejected a tensor of the prefill attention";
         return cudaErrorInvalidValue;
     }
@@ -616,9 +632,8 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
             max_len = std::max(max_len, lens_host[b0 + i]);
         }
         job.k_rows = std::min(l.capacity, (max_len + BKV - 1) / BKV * BKV);
-        const int64_t rows = (int64_t)nb * (l.kv_heads * (int64_t)job.k_rows + (int64_t)heads_q * n_new);
-        const unsigned blocks = (unsigned)std::min<int64_t>((rows + 15) / 16, 148 * 64);
-        prefill_rope_kernel<<<blocks, 256, 0, stream>>>(job);
+        const dim3 rope_grid((unsigned)((std::max(job.k_rows, n_new) + 63) / 64), (unsigned)(nb * (l.kv_heads + heads_q)));
+        prefill_rope_kernel<<<rope_grid, 256, 0, stream>>>(job);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         prm.n_new = n_new;
@@ -626,9 +641,11 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
         prm.g = g;
         prm.layer = layer;
         prm.batch0 = b0;
+        prm.batch_count = nb;
+        prm.q_tiles = (n_new + BQ - 1) / BQ;
         prm.out = static_cast<__nv_bfloat16*>(out);
         prm.status = status;
-        const dim3 grid((unsigned)((n_new + BQ - 1) / BQ), (unsigned)heads_q, (unsigned)nb);
+        const dim3 grid((unsigned)((int64_t)prm.q_tiles * heads_q * nb));
         prefill_attend_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(map_q, map_k, map_v, prm);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;

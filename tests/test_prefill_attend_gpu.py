@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from oracle import attention as oa
 from paper_2505_00570_b200 import binding as fk
 from paper_2505_00570_b200 import synth
@@ -174,3 +175,55 @@ def test_prefill_invalid_arguments(ctx):
     with pytest.raises(fk.FreqKVError) as e:
         ctx.attend_prefill(kf, torch.zeros_like(kf), 0, torch.zeros(1, 1, 10, 128, device="cuda"), [10])
     assert e.value.status == fk.ERR_UNSUPPORTED
+
+
+def test_chunkwise_prefill_interleaves_attention_and_compression(ctx):
+    """The loop of Section 3.3 on a small cache (256 rows, 4 sinks, 252 -> 126): every chunk is
+    appended, attended, and the full cache compressed before the next chunk goes in.  The oracle
+    runs its own fp64 pipeline (its own compressed caches, never the GPU's), so the comparison
+    covers the interplay of freqkv_append, freqkv_attend_prefill and freqkv_compress; the
+    tolerance grows with the number of compressions as in the stream tests."""
+    cap, sink, kept, total, H, G = 256, 4, 126, 900, 2, 2
+    rng = np.random.default_rng(20250500 + 31)
+    def ar1(n, d):  # low-frequency dominated rows, as the cache generator's channels
+        x = np.empty((n, d))
+        x[0] = rng.standard_normal(d)
+        for i in range(1, n):
+            x[i] = 0.9 * x[i - 1] + np.sqrt(1 - 0.81) * rng.standard_normal(d)
+        return x
+    toks_k = torch.tensor(np.stack([ar1(total, 128) for _ in range(H)])).to(torch.bfloat16)   # [H, T, d]
+    toks_v = torch.tensor(np.stack([ar1(total, 128) for _ in range(H)])).to(torch.bfloat16)
+    toks_q = torch.tensor(rng.standard_normal((H * G, total, 128))).to(torch.bfloat16)
+    k = torch.zeros(1, 1, H, cap, 128, device="cuda", dtype=torch.bfloat16)
+    v = torch.zeros_like(k)
+    ok = [np.zeros((cap, 128)) for _ in range(H)]   # the oracle's caches
+    ov = [np.zeros((cap, 128)) for _ in range(H)]
+    length, count, t0, worst = 0, 0, 0, 0.0
+    while t0 < total:
+        if length == cap:
+            length = ctx.compress(k, v, cap, kept, sink)
+            for h in range(H):
+                ok[h][sink:sink + kept] = oracle.compress_matrix(ok[h][sink:cap], kept)
+                ov[h][sink:sink + kept] = oracle.compress_matrix(ov[h][sink:cap], kept)
+            count += 1
+        n = min(total - t0, cap - length)
+        nk = toks_k[:, t0:t0 + n].reshape(1, 1, H, n, 128).contiguous().cuda()
+        nv = toks_v[:, t0:t0 + n].reshape(1, 1, H, n, 128).contiguous().cuda()
+        for h in range(H):
+            ok[h][length:length + n] = parity.to_f64(toks_k[h, t0:t0 + n])
+            ov[h][length:length + n] = parity.to_f64(toks_v[h, t0:t0 + n])
+        length = ctx.append(k, v, nk, nv, [length])[0]
+        q = toks_q[:, t0:t0 + n].reshape(1, H * G, n, 128).contiguous().cuda()
+        out = ctx.attend_prefill(k, v, 0, q, [length], rope_base=10000.0)
+        tol = TOL * (1 + count) ** 0.5
+        for i in sorted({0, n // 2, n - 1}):
+            for h in range(H):
+                want = oa.attend_decode(parity.to_f64(q[0, h * G:(h + 1) * G, i]), ok[h], ov[h], length - n + i + 1, 10000.0)
+                got = parity.to_f64(out[0, h * G:(h + 1) * G, i])
+                for g in range(G):
+                    err = parity.rel_l2(got[g], want[g])
+                    assert err <= tol, f"chunk at token {t0}, row {i}: relative L2 {err:.3e} after {count} compressions"
+                    worst = max(worst, err)
+        t0 += n
+    assert ctx.last_device_status() == fk.OK
+    assert count == oracle.compression_count(total, cap, sink, kept) and count >= 5

@@ -16,14 +16,18 @@
 //   pass 2, one CTA per (sequence, query head, 128 queries), 192 threads, two CTAs per SM (each
 //   holds half of the shared memory and of the tensor memory, so that one CTA's softmax overlaps
 //   the other's tensor-core work); the query tiles with the most keys are scheduled first:
-//     warp 0   TMA producer: the query tile once; per key tile of 64 rows the rotated keys and,
-//              straight from the cache through a 5-D tensor map, the values (two-stage rings);
+//     warp 0   TMA producer: the query tile once; per key tile of 64 rows the rotated keys (ring of
+//              three) and, straight from the cache through a 5-D tensor map, the values (ring of two);
 //     warp 1   MMA issuer: S = Q K_rot^T (fp16 in, fp32 in tensor memory, two S buffers so that
 //              the next tile's scores are computed while this tile's softmax runs), then
-//              O += P V (bf16 in; V is the MN-major operand, as it lies in the cache);
-//     warps 2-5 softmax, one query row per thread: read the row of S from tensor memory, causal
-//              mask on the diagonal tiles, running maximum and sum in base 2, weights rounded to
-//              bf16 into shared memory in the swizzled K-major operand layout.  O stays in tensor
+//              O += P V (bf16 in; P is read from tensor memory, V is the MN-major operand, as
+//              it lies in the cache);
+//     warps 2-5 softmax, one query row per thread (tensor-memory lane = row): read the row of S,
+//              causal mask on the diagonal tiles, running maximum and sum in base 2, weights rounded
+//              to bf16 and written back over the first 32 columns of the same S buffer (two
+//              per column, in key order: the A operand of the second product; the MMAs of one
+//              thread execute in order, so the scores that later overwrite the buffer cannot
+//              overtake the product that reads the weights).  O stays in tensor
 //              memory; it is rescaled (read, multiplied, written back) only when a row's maximum
 //              has grown by more than 2^8 since the reference was last moved -- the weights stay
 //              below 2^8 meanwhile, and the final division by the running sum makes the result
@@ -46,11 +50,10 @@ constexpr int BQ = 128;             // queries per CTA
 constexpr int BKV = 64;             // keys per tile
 constexpr int Q_SLAB = BQ * 128;    // bytes: 128 rows x 64 two-byte values, one 128-byte swizzle row each
 constexpr int Q_TILE = 2 * Q_SLAB;  // 128 queries x 128 channels
-constexpr int P_TILE = BQ * 128;    // 128 queries x 64 keys
 constexpr int KV_SLAB = BKV * 128;  // 64 rows x 64 channels
 constexpr int KV_TILE = 2 * KV_SLAB;
-constexpr int RING = 2;             // stages of the key ring and of the value ring
-constexpr int OFF_Q = 0, OFF_P = Q_TILE, OFF_K = OFF_P + P_TILE, OFF_V = OFF_K + RING * KV_TILE, OFF_BAR = OFF_V + RING * KV_TILE;
+constexpr int RING_K = 3, RING_V = 2;  // stages of the key ring (needed one tile earlier) and of the value ring
+constexpr int OFF_Q = 0, OFF_K = Q_TILE, OFF_V = OFF_K + RING_K * KV_TILE, OFF_BAR = OFF_V + RING_V * KV_TILE;
 constexpr int SMEM_USED = OFF_BAR + 256;
 // Two CTAs share an SM's 228 KB (1 KB of each CTA's share is reserved): 115712 bytes each at most.
 // The tiles need a 1024-byte aligned base; the slack left for aligning it is 768 bytes, and the
@@ -165,6 +168,17 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The same with the A operand in tensor memory: lane = row, 16-bit elements two per column in the
+// order of the contraction index.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // When every MMA issued so far has finished, arrive on the barrier.
@@ -300,16 +314,17 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     }
     uint8_t* aligned = smem_raw + (base - raw);
     const uint32_t bar0 = base + OFF_BAR;
-    // barriers: q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_free[2], p_ready, o_full
-    const uint32_t q_full = bar0;
-    auto k_full = [&](int s) { return bar0 + 8u * (1 + s); };
-    auto k_empty = [&](int s) { return bar0 + 8u * (3 + s); };
-    auto v_full = [&](int s) { return bar0 + 8u * (5 + s); };
-    auto v_empty = [&](int s) { return bar0 + 8u * (7 + s); };
-    auto s_full = [&](int s) { return bar0 + 8u * (9 + s); };
-    auto s_free = [&](int s) { return bar0 + 8u * (11 + s); };
-    const uint32_t p_ready = bar0 + 8u * 13, o_full = bar0 + 8u * 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + OFF_BAR + 8 * 15);
+    // barriers: q_full, p_ready, o_full, s_full[2], s_free[2], then per ring stage k_full, k_empty, v_full, v_empty
+    const uint32_t q_full = bar0, p_ready = bar0 + 8u, o_full = bar0 + 16u;
+    auto s_full = [&](int s) { return bar0 + 8u * (3 + s); };
+    auto s_free = [&](int s) { return bar0 + 8u * (5 + s); };
+    auto k_full = [&](int s) { return bar0 + 8u * (7 + s); };
+    auto k_empty = [&](int s) { return bar0 + 8u * (7 + RING_K + s); };
+    auto v_full = [&](int s) { return bar0 + 8u * (7 + 2 * RING_K + s); };
+    auto v_empty = [&](int s) { return bar0 + 8u * (7 + 2 * RING_K + RING_V + s); };
+    constexpr int N_BARRIERS = 7 + 2 * RING_K + 2 * RING_V;
+    static_assert(8 * N_BARRIERS + 8 <= 256, "barrier area");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + OFF_BAR + 8 * N_BARRIERS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -324,11 +339,15 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < RING; ++s) {
+        for (int s = 0; s < RING_K; ++s) {
             mbar_init(k_full(s), 1);
             mbar_init(k_empty(s), 1);
+        }
+        for (int s = 0; s < RING_V; ++s) {
             mbar_init(v_full(s), 1);
             mbar_init(v_empty(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(s_full(s), 1);
             mbar_init(s_free(s), 4);  // lane 0 of each softmax warp
         }
@@ -356,16 +375,15 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             tma_load_3d(base + OFF_Q, &map_q, q_full, 0, q0, q_slice);
             tma_load_3d(base + OFF_Q + Q_SLAB, &map_q, q_full, 64, q0, q_slice);
             for (int32_t t = 0; t < n_tiles; ++t) {
-                const int s = t % RING;
-                const uint32_t use = (uint32_t)(t / RING);
-                if (t >= RING && !mbar_wait(k_empty(s), (use - 1) & 1, abort_flag, prm.status)) break;
-                mbar_expect_tx(k_full(s), KV_TILE);
-                tma_load_3d(base + OFF_K + s * KV_TILE, &map_k, k_full(s), 0, t * BKV, k_slice);
-                tma_load_3d(base + OFF_K + s * KV_TILE + KV_SLAB, &map_k, k_full(s), 64, t * BKV, k_slice);
-                if (t >= RING && !mbar_wait(v_empty(s), (use - 1) & 1, abort_flag, prm.status)) break;
-                mbar_expect_tx(v_full(s), KV_TILE);
-                tma_load_5d(base + OFF_V + s * KV_TILE, &map_v, v_full(s), 0, t * BKV, h, prm.layer, prm.batch0 + b);
-                tma_load_5d(base + OFF_V + s * KV_TILE + KV_SLAB, &map_v, v_full(s), 64, t * BKV, h, prm.layer, prm.batch0 + b);
+                const int sk = t % RING_K, sv = t % RING_V;
+                if (t >= RING_K && !mbar_wait(k_empty(sk), ((uint32_t)(t / RING_K) - 1) & 1, abort_flag, prm.status)) break;
+                mbar_expect_tx(k_full(sk), KV_TILE);
+                tma_load_3d(base + OFF_K + sk * KV_TILE, &map_k, k_full(sk), 0, t * BKV, k_slice);
+                tma_load_3d(base + OFF_K + sk * KV_TILE + KV_SLAB, &map_k, k_full(sk), 64, t * BKV, k_slice);
+                if (t >= RING_V && !mbar_wait(v_empty(sv), ((uint32_t)(t / RING_V) - 1) & 1, abort_flag, prm.status)) break;
+                mbar_expect_tx(v_full(sv), KV_TILE);
+                tma_load_5d(base + OFF_V + sv * KV_TILE, &map_v, v_full(sv), 0, t * BKV, h, prm.layer, prm.batch0 + b);
+                tma_load_5d(base + OFF_V + sv * KV_TILE + KV_SLAB, &map_v, v_full(sv), 64, t * BKV, h, prm.layer, prm.batch0 + b);
             }
             if (*abort_flag) {  // let the copies in flight land before this CTA's shared memory goes away
                 const unsigned long long t0 = global_timer_ns();
@@ -377,9 +395,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         if (lane == 0) {
             bool alive = mbar_wait(q_full, 0, abort_flag, prm.status);
             auto issue_scores = [&](int32_t t) {
-                const int s = t % RING;
-                const uint32_t use = (uint32_t)(t / RING);
-                if (!mbar_wait(k_full(s), use & 1, abort_flag, prm.status)) return false;
+                const int s = t % RING_K;
+                if (!mbar_wait(k_full(s), (uint32_t)(t / RING_K) & 1, abort_flag, prm.status)) return false;
                 if (t >= 2 && !mbar_wait(s_free(t & 1), ((uint32_t)(t / 2) - 1) & 1, abort_flag, prm.status)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t qa = base + OFF_Q, ka = base + OFF_K + s * KV_TILE;
@@ -394,15 +411,16 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             if (alive) alive = issue_scores(0);
             for (int32_t t = 0; t < n_tiles && alive; ++t) {
                 if (t + 1 < n_tiles && !issue_scores(t + 1)) break;
-                const int s = t % RING;
+                const int s = t % RING_V;
                 if (!mbar_wait(p_ready, t & 1, abort_flag, prm.status)) break;
-                if (!mbar_wait(v_full(s), (t / RING) & 1, abort_flag, prm.status)) break;
+                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t pa = base + OFF_P, va = base + OFF_V + s * KV_TILE;
+                const uint32_t va = base + OFF_V + s * KV_TILE;
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk)  // 16 keys per instruction
-                    // P: K-major, one 64-key slab.  V: MN-major, 16 key rows = 2 KB per step, 64-channel slabs KV_SLAB apart.
-                    umma(tmem_o, smem_desc(pa + kk * 32, 16, 1024), smem_desc(va + kk * 2048, KV_SLAB, 1024), IDESC_PV, (t | kk) != 0);
+                    // P: in tensor memory over the first 32 columns of this tile's S buffer, 8 columns per step.
+                    // V: MN-major, 16 key rows = 2 KB per step, 64-channel slabs KV_SLAB apart.
+                    umma_ts(tmem_o, tmem_base + (t & 1) * BKV + kk * 8, smem_desc(va + kk * 2048, KV_SLAB, 1024), IDESC_PV, (t | kk) != 0);
                 umma_commit(o_full);
                 umma_commit(v_empty(s));
             }
@@ -413,11 +431,10 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         const uint32_t lane_bits = (uint32_t)(quarter * 32) << 16;
         const int32_t my_pos = pos0 + q0 + row;                      // keys up to this index are visible
         const int32_t warp_pos = pos0 + q0 + quarter * 32;           // the smallest position in this warp
-        uint8_t* p_row = aligned + OFF_P + row * 128;
         float m_ref = NEG_INF, l_run = 0.f;
         bool alive = true;
         for (int32_t t = 0; t < n_tiles; ++t) {
-            const int buf = t & 1, s = t % RING;
+            const int buf = t & 1, s = t % RING_V;
             const int32_t j0 = t * BKV;
             if (!mbar_wait(s_full(buf), (t / 2) & 1, abort_flag, prm.status)) { alive = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -473,12 +490,13 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             }
-            // weights into shared memory: K-major operand, 16-byte chunks XOR-swizzled by the row
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+            // weights over the first 32 columns of this tile's S buffer (bf16 pairs): the A operand of P V.  The scores that
+            // overwrite the buffer (tile t + 2) are issued behind that P V, and one thread's MMAs execute in order.
+            tmem_st32(tmem_base + lane_bits + buf * BKV, pk);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (j0 + BKV > len) {  // value rows past the cache length are stale: make them zeros
-                if (!mbar_wait(v_full(s), (t / RING) & 1, abort_flag, prm.status)) { alive = false; break; }
+                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status)) { alive = false; break; }
                 if (row < BKV && j0 + row >= len) {
                     uint8_t* v_row = aligned + OFF_V + s * KV_TILE + row * 128;
 #pragma unroll
@@ -487,8 +505,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                         *reinterpret_cast<uint4*>(v_row + KV_SLAB + c * 16) = make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> the tensor core's reads
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> the tensor core's reads
             mbar_arrive(p_ready);
         }
         if (alive && mbar_wait(o_full, (n_tiles - 1) & 1, abort_flag, prm.status)) {

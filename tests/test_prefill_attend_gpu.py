@@ -227,3 +227,12 @@ def test_chunkwise_prefill_interleaves_attention_and_compression(ctx):
         t0 += n
     assert ctx.last_device_status() == fk.OK
     assert count == oracle.compression_count(total, cap, sink, kept) and count >= 5
+
+
+def test_prefill_more_sequences_than_one_launch_takes(ctx):
+    """130 short sequences: the lengths travel as kernel arguments, 128 per launch."""
+    w = workload(130, 1, 1, 96, seed=29)
+    k, v = synth.make_cache(w, "cuda")
+    lens = [96 - (b % 50) for b in range(130)]
+    q = queries(130, 2, 7, 11)
+    check(ctx, k, v, 0, q, lens, 10000.0, heads=[(0, 0), (127, 0), (128, 0), (129, 0)])

@@ -403,14 +403,14 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 
-def run_prefill_attend(args, ctx, fk, synth, dev, peaks):
-    """Chunk-wise prefilling attention (Section 3.3) of one 7B-shaped layer: the 2046 tokens that
-    refill the cache after a compression attend causally to 4 sinks + 2046 compressed rows + the
-    chunk.  One freqkv_attend_prefill call per step, layers alternating."""
-    B, H, G, cap, base = 1, 32, 1, 4096, 10000.0
+def run_prefill_attend(args, ctx, fk, synth, name, dev, peaks):
+    """Chunk-wise prefilling attention (Section 3.3) of one layer: the tokens that refill the cache
+    after a compression (2046 on the 7B shape, 4094 on the 8B shape) attend causally to 4 sinks +
+    the compressed rows + the chunk.  One freqkv_attend_prefill call per step, layers alternating."""
+    B, H, G, cap, base = {"prefill_attend_7b": (1, 32, 1, 4096, 10000.0), "prefill_attend_8b": (1, 8, 4, 8192, 500000.0)}[name]
     n_new = cap - 4 - (cap - 4) // 2
     layers = 4
-    w = synth.Workload("prefill_attend_7b", B, layers, H, 128, cap, torch.bfloat16, 4, 0.9, 2, synth.BASE_SEED + 8)
+    w = synth.Workload(name, B, layers, H, 128, cap, torch.bfloat16, 4, 0.9, 2, synth.BASE_SEED + 8)
     k, v = synth.make_cache(w, dev)
     gen = torch.Generator(device=dev)
     gen.manual_seed(w.seed + 1)
@@ -440,7 +440,7 @@ def run_prefill_attend(args, ctx, fk, synth, dev, peaks):
     return {"metric": "prefill attention TFLOP/s (causal pairs only)", "value": flops_per_call / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
             "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "prefill_attend_7b", "batch": B, "kv_heads": H, "q_heads_per_kv": G, "head_dim": 128,
+            "config": {"workload": name, "batch": B, "kv_heads": H, "q_heads_per_kv": G, "head_dim": 128,
                        "cache_len": cap, "chunk": n_new, "rope_base": base,
                        "step": "one freqkv_attend_prefill call over one layer", "l2": "%d layers alternate" % layers},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
@@ -522,13 +522,13 @@ def main():
             print(json.dumps(run_spectrum(args, ctx, fk, synth, torch.device("cuda", local_rank), load_peaks())), flush=True)
             ctx.close()
         return
-    if args.workload == "prefill_attend_7b":          # side workload: chunk-wise prefilling attention
+    if args.workload in ("prefill_attend_7b", "prefill_attend_8b"):  # side workload: chunk-wise prefilling attention
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
         if rank == 0:
             torch.cuda.set_device(local_rank)
             ctx = fk.Context(local_rank)
-            print(json.dumps(run_prefill_attend(args, ctx, fk, synth, torch.device("cuda", local_rank), load_peaks())), flush=True)
+            print(json.dumps(run_prefill_attend(args, ctx, fk, synth, args.workload, torch.device("cuda", local_rank), load_peaks())), flush=True)
             ctx.close()
         return
     if args.workload in ("attend_7b", "attend_8b"):   # side workload: the step after the compression path

@@ -236,3 +236,21 @@ def test_prefill_more_sequences_than_one_launch_takes(ctx):
     lens = [96 - (b % 50) for b in range(130)]
     q = queries(130, 2, 7, 11)
     check(ctx, k, v, 0, q, lens, 10000.0, heads=[(0, 0), (127, 0), (128, 0), (129, 0)])
+
+
+@pytest.mark.parametrize("G", [3, 8])
+def test_prefill_other_group_sizes(ctx, G):
+    """Any number of query heads per KV head: each query head is its own CTA column."""
+    w = workload(1, 1, 2, 192, seed=30)
+    k, v = synth.make_cache(w, "cuda")
+    check(ctx, k, v, 0, queries(1, 2 * G, 40, 12 + G), [150], 10000.0, tokens=(0, 17, 39))
+
+
+def test_prefill_smallest_caches(ctx):
+    """One token in a cache of one row; a chunk that is a whole cache whose length is no multiple of the tile sizes."""
+    w = workload(1, 1, 1, 128, seed=31)
+    k, v = synth.make_cache(w, "cuda")
+    q1 = queries(1, 1, 1, 13)
+    out = ctx.attend_prefill(k, v, 0, q1, [1], rope_base=10000.0)
+    assert torch.equal(out[0, 0, 0], v[0, 0, 0, 0])
+    check(ctx, k, v, 0, queries(1, 1, 100, 14), [100], 10000.0, tokens=(0, 1, 63, 64, 65, 99))

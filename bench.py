@@ -399,7 +399,7 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": "copy, of " + peaks["source"],
                          "kernel": ("attend_mma_kernel" if G >= 2 else "attend_partial_kernel") + " + attend_merge_kernel",
                          "kernel_ms": kernel_ms,
-                         "traffic": None},
+                         "traffic": load_traffic(name, "attend")},
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 
@@ -445,7 +445,7 @@ def run_prefill_attend(args, ctx, fk, synth, name, dev, peaks):
                        "step": "one freqkv_attend_prefill call over one layer", "l2": "%d layers alternate" % layers},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                          "peak_kind": "cuBLAS bf16 burst, of " + peaks["source"],
-                         "kernel": "prefill_rope_kernel + prefill_attend_kernel", "kernel_ms": kernel_ms, "traffic": None},
+                         "kernel": "prefill_rope_kernel + prefill_attend_kernel", "kernel_ms": kernel_ms, "traffic": load_traffic(name, "attend")},
             "cpu_baseline": None, "e2e": None, "gpu_launches": 2 * args.steps}
 
 

@@ -16,8 +16,8 @@
 //   pass 2, one CTA per (sequence, query head, 128 queries), 192 threads, two CTAs per SM (each
 //   holds half of the shared memory and of the tensor memory, so that one CTA's softmax overlaps
 //   the other's tensor-core work); the query tiles with the most keys are scheduled first:
-//     warp 0   TMA producer: the query tile once; per key tile of 64 rows the rotated keys (ring of
-//              three) and, straight from the cache through a 5-D tensor map, the values (ring of two);
+//     warp 0   TMA producer: the query tile once; per key tile of 64 rows the rotated keys and,
+//              straight from the cache through a 5-D tensor map, the values (two-stage rings);
 //     warp 1   MMA issuer: S = Q K_rot^T (fp16 in, fp32 in tensor memory, two S buffers so that
 //              the next tile's scores are computed while this tile's softmax runs), then
 //              O += P V (bf16 in; P is read from tensor memory, V is the MN-major operand, as
@@ -52,14 +52,11 @@ constexpr int Q_SLAB = BQ * 128;    // bytes: 128 rows x 64 two-byte values, one
 constexpr int Q_TILE = 2 * Q_SLAB;  // 128 queries x 128 channels
 constexpr int KV_SLAB = BKV * 128;  // 64 rows x 64 channels
 constexpr int KV_TILE = 2 * KV_SLAB;
-constexpr int RING_K = 3, RING_V = 2;  // stages of the key ring (needed one tile earlier) and of the value ring
+constexpr int RING_K = 2, RING_V = 2;  // stages of the key ring and of the value ring (a third key stage measured no faster)
 constexpr int OFF_Q = 0, OFF_K = Q_TILE, OFF_V = OFF_K + RING_K * KV_TILE, OFF_BAR = OFF_V + RING_V * KV_TILE;
 constexpr int SMEM_USED = OFF_BAR + 256;
-// Two CTAs share an SM's 228 KB (1 KB of each CTA's share is reserved): 115712 bytes each at most.
-// The tiles need a 1024-byte aligned base; the slack left for aligning it is 768 bytes, and the
-// kernel checks that it was enough (a base that is 1024-aligned already needs none).
-constexpr int SMEM_BYTES = 115712;
-static_assert(SMEM_USED <= SMEM_BYTES, "the tiles of a CTA must leave room for a second CTA on the SM");
+constexpr int SMEM_BYTES = SMEM_USED + 1024;  // + slack for aligning the base to 1024 bytes
+static_assert(2 * (SMEM_BYTES + 1024) <= 233472, "two CTAs per SM (1 KB of each CTA's share is reserved)");
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 256;      // S buffers in columns 0..63 and 64..127, O in 128..255
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
@@ -308,10 +305,6 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
-    if (base - raw + SMEM_USED > SMEM_BYTES) {     // uniform over the CTA; nothing has been set up yet
-        if (threadIdx.x == 0) atomicOr(prm.status, PREFILL_ERR_WAIT);
-        return;
-    }
     uint8_t* aligned = smem_raw + (base - raw);
     const uint32_t bar0 = base + OFF_BAR;
     // barriers: q_full, p_ready, o_full, s_full[2], s_free[2], then per ring stage k_full, k_empty, v_full, v_empty

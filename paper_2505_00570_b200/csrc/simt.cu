@@ -147,6 +147,23 @@ __global__ void append_kernel(CacheView view, int32_t batch, AppendLens lens, in
     }
 }
 
+// One new row per matrix (a decode step): one thread per 16 bytes, 32-bit index arithmetic, no grid-stride loop.
+__global__ void __launch_bounds__(256) append_one_kernel(CacheView view, int32_t batch, AppendLens lens, int32_t elt_size,
+                                                         const uint4* __restrict__ new_k, const uint4* __restrict__ new_v)
+{
+    const uint32_t vec_per_row = (uint32_t)(view.head_dim * elt_size / 16);
+    const uint32_t per_tensor = (uint32_t)(batch * view.layers * view.kv_heads) * vec_per_row;
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 2 * per_tensor) return;
+    const uint32_t tensor = i >= per_tensor, j = i - tensor * per_tensor;
+    const uint32_t vcol = j % vec_per_row, idx = j / vec_per_row;
+    const uint32_t b = idx / (uint32_t)(view.layers * view.kv_heads);
+    const uint4 val = __ldg((tensor ? new_v : new_k) + j);
+    const int64_t off = matrix_offset(view, (int32_t)idx) + (int64_t)lens.len[b] * view.stride_token;
+    char* dst = static_cast<char*>(tensor_base(view, (int32_t)tensor)) + off * elt_size;
+    reinterpret_cast<uint4*>(dst)[vcol] = val;
+}
+
 // Many new rows per matrix (prefill chunks): one block column per matrix, so that the matrix
 // arithmetic is done once per thread and each thread then moves four 16-byte vectors per round,
 // loads first.  Block (x, y): matrix x (K matrices first, then V), y-th share of its vectors.
@@ -319,6 +336,8 @@ cudaError_t launch_append(const CacheView& view, int32_t dtype, int32_t batch, c
         if (mat_vecs >= 4096 && mat_vecs < ((int64_t)1 << 31) && mats2 < ((int64_t)1 << 31)) {
             const unsigned gy = (unsigned)std::min<int64_t>((mat_vecs + 1023) / 1024, 64);
             append_rows_kernel<<<dim3((unsigned)mats2, gy), 256, 0, stream>>>(sub, nb, lens, n_new, elt, nk, nv);
+        } else if (n_new == 1 && 2 * nb * seq_vecs < ((int64_t)1 << 31)) {
+            append_one_kernel<<<(unsigned)((2 * nb * seq_vecs + 255) / 256), 256, 0, stream>>>(sub, nb, lens, elt, nk, nv);
         } else {
             append_kernel<<<grid_for(2 * nb * seq_vecs, 256), 256, 0, stream>>>(sub, nb, lens, n_new, elt, nk, nv);
         }

@@ -21,7 +21,8 @@
 // factor) butterfly at a time per thread, held in registers: the forward one as decimation in
 // time on digit-reversed input -- the load phase puts every element where that order wants it --
 // the inverse one as decimation in frequency, whose digit-reversed output the store phase reads
-// back in row order.  Twiddles come from an fp64-built table through the read-only cache.
+// back in row order.  The twiddle of a butterfly is computed (sincospif of an exactly scaled
+// index); the factors of the DCT spectrum and of the inverse's pre-twiddle come from fp64-built tables.
 // Indices are padded (see pad()) so that the passes meet few shared-memory bank conflicts.
 #include <cuda.h>
 
@@ -169,7 +170,6 @@ __device__ __forceinline__ void fft_pass(float2* s, int log_n, int seq_stride, i
     constexpr int STEP = LOG_S == 0 ? 1 : LOG_S == 4 ? 17 : S + (S >> 4) + (S >> 8);
     const int log_bf = log_n - log_r;  // butterflies per sequence
     const int total = pairs << log_bf;
-    const int tw_shift = log_table - LOG_S - log_r;
     for (int g = tid; g < total; g += THREADS) {
         const int pair = g >> log_bf, j = g & ((1 << log_bf) - 1), k = j & (S - 1);
         float2* x = s + pair * seq_stride + pad(((j >> LOG_S) << (LOG_S + log_r)) + k);
@@ -179,7 +179,10 @@ __device__ __forceinline__ void fft_pass(float2* s, int log_n, int seq_stride, i
         if constexpr (LOG_S > 0) {
             // w^q for q = 1 .. R-1 from one table entry: w^2 and w^3 by products, the rest as
             // w^(4a+b) = (w^4)^a w^b, so that no power is more than three products away from the table
-            float2 w1 = __ldg(W + (k << tw_shift));
+            // w = exp(-2 pi i k / (S R)), computed (an exact power-of-two scaling of k, then sincospif): a table
+            // entry per butterfly would cost one scattered 8-byte global load per lane on the load/store pipe
+            float2 w1;
+            sincospif(-(float)k * (2.0f / (float)(S << log_r)), &w1.y, &w1.x);
             if (INV) w1.y = -w1.y;
             if (!INV) twiddle_all<R>(v, w1);
             SmallFft<R, INV>::run(v);

@@ -618,8 +618,10 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
         *error = "cuTensorMapEncodeTiled rejected a tensor of the prefill attention";
         return cudaErrorInvalidValue;
     }
-    for (int32_t b0 = 0; b0 < l.batch; b0 += PREFILL_MAX_BATCH) {
-        const int32_t nb = std::min(PREFILL_MAX_BATCH, l.batch - b0);
+    // sequences per launch: their lengths travel as kernel arguments, and the pre-pass puts one slice per grid row
+    const int32_t per_launch = std::max(1, std::min(PREFILL_MAX_BATCH, 65535 / (l.kv_heads + l.kv_heads * g)));
+    for (int32_t b0 = 0; b0 < l.batch; b0 += per_launch) {
+        const int32_t nb = std::min(per_launch, l.batch - b0);
         int32_t max_len = 0;
         RopeJob job;
         job.k = static_cast<const __nv_bfloat16*>(k) + (int64_t)layer * l.stride_layer;

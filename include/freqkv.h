@@ -230,7 +230,8 @@ freqkv_status freqkv_attend_decode(freqkv_ctx* ctx, const freqkv_layout* layout,
  * range, n_new < 1, a length outside [n_new, capacity], NaN scale or base), UNSUPPORTED (fp32
  * caches, head_dim != 128, misaligned pointers, layout rules), ALLOC, CUDA.  The context keeps
  * two scratch buffers (rotated keys of one layer, rotated queries of one chunk) and the cos/sin
- * table.  A barrier wait inside the kernel that runs out (2 s) ends the kernel and shows up in
+ * table; they are allocated, or grown after a device synchronisation, by the first call that
+ * needs them (so make that call before any stream capture).  A barrier wait inside the kernel that runs out (2 s) ends the kernel and shows up in
  * freqkv_last_device_status as TIMEOUT. */
 freqkv_status freqkv_attend_prefill(freqkv_ctx* ctx, const freqkv_layout* layout, const void* k, const void* v,
                                     int32_t layer, const void* q, void* out, int32_t q_heads_per_kv, int32_t n_new,

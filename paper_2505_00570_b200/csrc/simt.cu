@@ -222,24 +222,25 @@ __global__ void decode_set_lens_kernel(int32_t* lens, int32_t batch, int32_t val
 }
 
 // One new row per matrix, written at the sequence's device-resident length (full sequences are skipped).
-__global__ void decode_append_kernel(CacheView view, int32_t batch, const int32_t* __restrict__ lens, int32_t capacity,
-                                     int32_t elt_size, const uint4* __restrict__ new_k, const uint4* __restrict__ new_v)
+// One thread per 16 bytes; 32-bit index arithmetic when the count allows it.
+template <typename I>
+__global__ void __launch_bounds__(256) decode_append_kernel(CacheView view, int32_t batch, const int32_t* __restrict__ lens,
+                                                            int32_t capacity, int32_t elt_size, const uint4* __restrict__ new_k,
+                                                            const uint4* __restrict__ new_v)
 {
-    const int32_t vec_per_row = view.head_dim * elt_size / 16;
-    const int32_t mats = batch * view.layers * view.kv_heads;
-    const int64_t per_tensor = (int64_t)mats * vec_per_row;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < 2 * per_tensor;
-         i += (int64_t)gridDim.x * blockDim.x) {
-        const int32_t tensor = i >= per_tensor;
-        const int64_t j = i - tensor * per_tensor;
-        const int32_t vcol = (int32_t)(j % vec_per_row), idx = (int32_t)(j / vec_per_row);
-        const int32_t b = idx / (view.layers * view.kv_heads);
-        const int32_t len = lens[b];
-        if (len >= capacity) continue;
-        const int64_t off = matrix_offset(view, idx) + (int64_t)len * view.stride_token;
-        char* dst = static_cast<char*>(tensor_base(view, tensor)) + off * elt_size;
-        reinterpret_cast<uint4*>(dst)[vcol] = (tensor ? new_v : new_k)[j];
-    }
+    const I vec_per_row = (I)(view.head_dim * elt_size / 16);
+    const I per_tensor = (I)batch * (I)(view.layers * view.kv_heads) * vec_per_row;
+    const I i = (I)blockIdx.x * (I)blockDim.x + (I)threadIdx.x;
+    if (i >= 2 * per_tensor) return;
+    const I tensor = i >= per_tensor ? 1 : 0, j = i - tensor * per_tensor;
+    const I vcol = j % vec_per_row, idx = j / vec_per_row;
+    const int32_t b = (int32_t)(idx / (I)(view.layers * view.kv_heads));
+    const int32_t len = lens[b];
+    if (len >= capacity) return;
+    const uint4 val = __ldg((tensor ? new_v : new_k) + j);
+    const int64_t off = matrix_offset(view, (int32_t)idx) + (int64_t)len * view.stride_token;
+    char* dst = static_cast<char*>(tensor_base(view, (int32_t)tensor)) + off * elt_size;
+    reinterpret_cast<uint4*>(dst)[vcol] = val;
 }
 
 __global__ void decode_advance_kernel(int32_t* lens, int32_t batch, int32_t capacity)
@@ -308,8 +309,12 @@ cudaError_t launch_decode_append(const CacheView& view, int32_t dtype, int32_t b
 {
     const int32_t elt = (int32_t)dtype_size(dtype);
     const int64_t vecs = (int64_t)2 * batch * view.layers * view.kv_heads * (view.head_dim * elt / 16);
-    decode_append_kernel<<<grid_for(vecs, 256), 256, 0, stream>>>(view, batch, lens, capacity, elt,
-                                                                  static_cast<const uint4*>(new_k),
+    const unsigned blocks = (unsigned)((vecs + 255) / 256);
+    if (vecs < ((int64_t)1 << 31))
+        decode_append_kernel<uint32_t><<<blocks, 256, 0, stream>>>(view, batch, lens, capacity, elt, static_cast<const uint4*>(new_k),
+                                                                  static_cast<const uint4*>(new_v));
+    else
+        decode_append_kernel<uint64_t><<<blocks, 256, 0, stream>>>(view, batch, lens, capacity, elt, static_cast<const uint4*>(new_k),
                                                                   static_cast<const uint4*>(new_v));
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

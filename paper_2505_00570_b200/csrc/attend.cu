@@ -622,6 +622,9 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(const float* __restri
 {
     const int64_t head = blockIdx.x;
     const int c = threadIdx.x;
+    // launched with programmatic stream serialization: the blocks may start while the kernel that
+    // writes the partials is still draining; wait here until that grid has completed and its writes are visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float mn = NEG, sum = 0.f, acc = 0.f;
 #pragma unroll 8
     for (int s = 0; s < splits; ++s) {
@@ -756,12 +759,20 @@ cudaError_t launch_attend(const freqkv_layout& l, const void* k, const void* v, 
         if (e != cudaSuccess) return e;
     }
     const int64_t heads_total = (int64_t)l.batch * l.kv_heads * g;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)heads_total);
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // let the launch overlap the tail of the kernel before it
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const float* partial_in = partial;
     if (l.dtype == FREQKV_F32)
-        attend_merge_kernel<float><<<(unsigned)heads_total, 128, 0, stream>>>(partial, splits, heads_total, static_cast<float*>(out));
-    else
-        attend_merge_kernel<__nv_bfloat16><<<(unsigned)heads_total, 128, 0, stream>>>(partial, splits, heads_total,
-                                                                                  static_cast<__nv_bfloat16*>(out));
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, attend_merge_kernel<float>, partial_in, splits, heads_total, static_cast<float*>(out));
+    return cudaLaunchKernelEx(&cfg, attend_merge_kernel<__nv_bfloat16>, partial_in, splits, heads_total,
+                              static_cast<__nv_bfloat16*>(out));
 }
 
 }  // namespace freqkv

@@ -364,6 +364,9 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const int32_t q_slice = (prm.batch0 + b) * heads_q + hq, k_slice = (prm.batch0 + b) * prm.kv_heads + h;
+            // launched with programmatic stream serialization: the set-up above may run while pass 1 drains; its
+            // output (read only through these loads) is complete and visible after this wait
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             mbar_expect_tx(q_full, Q_TILE);
             tma_load_3d(base + OFF_Q, &map_q, q_full, 0, q0, q_slice);
             tma_load_3d(base + OFF_Q + Q_SLAB, &map_q, q_full, 64, q0, q_slice);
@@ -659,8 +662,17 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
         prm.out = static_cast<__nv_bfloat16*>(out);
         prm.status = status;
         const dim3 grid((unsigned)((int64_t)prm.q_tiles * heads_q * nb));
-        prefill_attend_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(map_q, map_k, map_v, prm);
-        e = cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // let the launch overlap the tail of pass 1
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, prefill_attend_kernel, map_q, map_k, map_v, prm);
         if (e != cudaSuccess) return e;
         *kernels_launched += 2;
     }

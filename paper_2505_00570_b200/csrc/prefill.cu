@@ -11,8 +11,8 @@
 //   pass 1 (CUDA cores, one read of the layer's keys and of the queries): rotate the keys of the
 //     layer and the queries of the chunk, the queries also scaled by scale * log2(e), and round
 //     them to fp16 into scratch (fp16 rather than bf16: three more mantissa bits keep the error of
-//     the scores a quarter of bf16's).  Key rows from the length to the next multiple of 128 are
-//     written as zeros.
+//     the scores a quarter of bf16's).  Key rows from the length to the next multiple of the key
+//     tile are written as zeros.
 //   pass 2, one CTA per (sequence, query head, 128 queries), 192 threads, two CTAs per SM (each
 //   holds half of the shared memory and of the tensor memory, so that one CTA's softmax overlaps
 //   the other's tensor-core work); the query tiles with the most keys are scheduled first:

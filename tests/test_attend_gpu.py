@@ -128,3 +128,13 @@ def test_attend_invalid_arguments(ctx):
     with pytest.raises(fk.FreqKVError) as e:
         ctx.attend_decode(k64, torch.zeros_like(k64), 0, torch.zeros(1, 1, 64, device="cuda", dtype=torch.bfloat16), [10])
     assert e.value.status == fk.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_attend_more_sequences_than_one_launch_takes(ctx, G):
+    """131 short sequences: the lengths travel as kernel arguments, 128 per launch, and one merge
+    launch follows the last of them."""
+    w = workload(131, 1, 1, 96, torch.bfloat16, seed=16)
+    k, v = synth.make_cache(w, "cuda")
+    lens = [96 - (b % 60) for b in range(131)]
+    check(ctx, k, v, 0, queries(131, G, torch.bfloat16, 17 + G), lens, 10000.0, heads=[(0, 0), (1, 0), (127, 0), (128, 0), (130, 0)])

@@ -654,11 +654,21 @@ def main():
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": "copy, of " + peaks["source"]}
     elif chosen == fk.GEMM:
         achieved = nums["folded_flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": "sustained, of " + peaks["source"],
+        # the burst figure is the denominator for a timed region of under a second, the sustained
+        # one (power cap reached) for longer loops; both fractions are printed
+        burst = ms_total < 1000.0
+        peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+        fold_ms = max(compress_ms - kernel_ms * per_call, 0.0)
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "peak_kind": ("burst" if burst else "sustained") + ", of " + peaks["source"],
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                 "flops_per_launch": nums["folded_flops_per_launch"],
-                "dense_equivalent_flops_per_launch": nums["projection_flops_per_launch"]}
+                "dense_equivalent_flops_per_launch": nums["projection_flops_per_launch"],
+                # the fold pass the kernel cannot run without: its time (compress call minus the
+                # timed kernel) and the bytes it moves (every non-sink row read once, written once)
+                "fold_ms": fold_ms, "fold_bytes": 2 * nums["matrices"] * (cache_len - sink) * w.head_dim * 2,
+                "frac_of_burst_peak_whole_call": nums["folded_flops"] / (compress_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
     elif chosen == fk.FDCT:
         achieved = nums["algorithmic_bytes_per_launch"] / (kernel_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -13,8 +13,12 @@
  *    reallocates them.  `lens`, `kept_len` arrays and layout structs are HOST memory.
  *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *    Calls enqueue work on it and return without synchronising, unless stated otherwise.
- *  - Every function returns a freqkv_status; on any status other than FREQKV_OK nothing was
- *    enqueued and no caller memory was modified.  No C++ exception crosses the boundary.
+ *  - Every function returns a freqkv_status.  Arguments are validated in full before anything
+ *    is enqueued: on INVALID_ARG, UNSUPPORTED and CAPACITY nothing was enqueued and no caller
+ *    memory was modified.  FREQKV_ERR_ALLOC / FREQKV_ERR_CUDA can also come from the middle of
+ *    a call that works in several passes (large caches, ragged batches, host buffers): passes
+ *    enqueued before the failure still run, so the rows a compression rewrites are then
+ *    undefined (everything else keeps its bytes).  No C++ exception crosses the boundary.
  *  - A context belongs to one device and must not be used from two threads at once.  Its work
  *    areas are shared by its calls: a call enqueued on another stream than the previous one first
  *    waits (on the device) for that one, so calls on one context never overlap on the GPU; use
@@ -250,17 +254,20 @@ freqkv_status freqkv_get_timing(freqkv_ctx* ctx, int64_t* transform_launches, do
 /* Compression for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of freqkv_compress, same definition, same result.)
  *
- * Who needs it: code that runs where cudaMalloc is not allowed or not safe -- inside a CUDA
- * stream capture, under a lock that an allocation's implicit synchronisation could deadlock
- * against, in a serving loop whose device-memory budget is frozen, or inside a host framework
- * that owns all device memory.  freqkv_compress does not fit there: its context, its plan and
- * its staging buffer all come from cudaMalloc.
+ * Who needs it: code that runs where cudaMalloc is not allowed or not safe -- under a lock that
+ * an allocation's implicit device synchronisation could deadlock against, in a serving loop
+ * whose device-memory budget is frozen, or inside a host framework that owns all device memory.
+ * freqkv_compress does not fit there: its context, its plan and its staging buffer all come
+ * from cudaMalloc.
  *
  * What it does: the CUDA-core (SIMT) projection of freqkv_compress with its two work areas --
  * the fp32 projection basis and the staging area for compressed rows -- placed in fixed arrays
  * inside the library image instead of allocated memory.  No context is needed; `k` and `v` are
  * device pointers exactly as for freqkv_compress and the arrays of the device that owns them are
- * used.  The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ * used: both must be plain device allocations of ONE device (INVALID_ARG for host or managed
+ * memory, or when k and v live on different devices).  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating call, so free device memory is the same before and after it.
+ * If a launch fails (FREQKV_ERR_CUDA) the groups of matrices enqueued before it still run.
  *
  * Limits (FREQKV_ERR_UNSUPPORTED beyond them, nothing enqueued): with n_in = cache_len - sink,
  *   roundup(n_in, 64) * roundup(kept_len, 64) <= FREQKV_NOALLOC_MAX_BASIS_ELEMS   (1 Mi entries),
@@ -278,6 +285,17 @@ freqkv_status freqkv_get_timing(freqkv_ctx* ctx, int64_t* transform_launches, do
 #define FREQKV_NOALLOC_STAGING_BYTES (4u << 20)
 freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, void* k, void* v, int32_t cache_len,
                                       int32_t kept_len, int32_t sink, void* cuda_stream);
+
+/* Every wait of a tensor-core kernel on one of its barriers is bounded; this sets the bound for
+ * later launches of this context (default 2 s; at least 1000 ns).  A wait that runs out ends the
+ * kernel and is reported by freqkv_last_device_status as FREQKV_ERR_TIMEOUT. */
+freqkv_status freqkv_set_wait_limit(freqkv_ctx* ctx, int64_t nanoseconds);
+
+/* Self-test of that give-up path: enqueues a one-thread kernel that waits, with the kernels' own
+ * bounded wait, on a barrier nothing ever arrives on.  After `nanoseconds` (1000 .. 1e9) it gives
+ * up, sets its bit in the status word and returns -- the next freqkv_last_device_status reports
+ * FREQKV_ERR_TIMEOUT, the one after that FREQKV_OK, and the context stays usable. */
+freqkv_status freqkv_selftest_bounded_wait(freqkv_ctx* ctx, int64_t nanoseconds, void* cuda_stream);
 
 /* Synchronise `cuda_stream`, then read and clear the device status word.  FREQKV_OK unless a
  * kernel's bounded wait (mbarrier / flag) ran out, in which case the affected output rows are

@@ -30,6 +30,7 @@ EXPORTS = [
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
     "freqkv_attend_prefill", "freqkv_check_attend_prefill",
     "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
+    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -93,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.freqkv_attend_prefill.argtypes = [c_void_p, LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32,
                                             I32P, ctypes.c_float, ctypes.c_float, c_void_p]
         L.freqkv_check_attend_prefill.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, I32P]
+        L.freqkv_set_wait_limit.argtypes = [c_void_p, c_int64]
+        L.freqkv_selftest_bounded_wait.argtypes = [c_void_p, c_int64, c_void_p]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -169,8 +172,8 @@ def _stream_ptr(stream) -> int:
 
 def compress_noalloc(k: torch.Tensor, v: torch.Tensor, cache_len: int, kept_len: int, sink: int, stream=None) -> int:
     """``freqkv_compress_noalloc``: in-place compression without a context and without any
-    device allocation, for callers that cannot call cudaMalloc (stream capture, frozen memory
-    budgets).  Small shapes only: see the limits in ``include/freqkv.h``.  Returns the new
+    device allocation, for callers that cannot call cudaMalloc (frozen memory budgets,
+    frameworks that own all device memory).  Small shapes only: see the limits in ``include/freqkv.h``.  Returns the new
     cache length; raises FreqKVError (ERR_UNSUPPORTED beyond the size limits)."""
     lay = layout_of(k)
     if tuple(v.shape) != tuple(k.shape) or v.stride() != k.stride() or v.dtype != k.dtype:
@@ -398,6 +401,16 @@ class Context:
         n, ms, k = c_int64(0), ctypes.c_double(0.0), c_int64(0)
         self._check(lib().freqkv_get_timing(self._h, ctypes.byref(n), ctypes.byref(ms), ctypes.byref(k)), "freqkv_get_timing")
         return n.value, ms.value, k.value
+
+    def set_wait_limit(self, nanoseconds: int):
+        self._check(lib().freqkv_set_wait_limit(self._h, nanoseconds), "freqkv_set_wait_limit")
+
+    def selftest_bounded_wait(self, nanoseconds: int, stream=None):
+        """Enqueue the one-thread kernel whose bounded barrier wait runs out after `nanoseconds`."""
+        self._check(lib().freqkv_selftest_bounded_wait(self._h, nanoseconds, _stream_ptr(stream)), "freqkv_selftest_bounded_wait")
+
+    def last_error(self) -> str:
+        return lib().freqkv_last_error(self._h).decode()
 
     def last_device_status(self, stream=None) -> int:
         return lib().freqkv_last_device_status(self._h, _stream_ptr(stream))

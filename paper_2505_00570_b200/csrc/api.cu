@@ -309,6 +309,31 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
     return FREQKV_OK;
 }
 
+size_t basis_device_bytes(const Basis& b)
+{
+    return (b.f32 ? (size_t)b.ld * b.rows_pad * 4 : 0) + (b.fold ? (size_t)2 * b.fold_ld * b.fold_rows_pad * 2 : 0) +
+           (b.dense ? (size_t)256 * b.ld * 2 : 0);
+}
+
+// Remove the plan of (n_in, n_keep, first) from the cache without freeing it: the caller owns its
+// device memory from now on (later calls on the context build a fresh one).
+void disown_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t first)
+{
+    auto it = ctx->bases.find(std::make_tuple(n_in, n_keep, first));
+    if (it == ctx->bases.end()) return;
+    const size_t bytes = basis_device_bytes(it->second);
+    ctx->basis_bytes = ctx->basis_bytes > bytes ? ctx->basis_bytes - bytes : 0;
+    ctx->bases.erase(it);
+}
+
+void free_basis(Basis* b)
+{
+    if (b->f32) cudaFree(b->f32);
+    if (b->fold) cudaFree(b->fold);
+    if (b->dense) cudaFree(b->dense);
+    *b = Basis();
+}
+
 freqkv_status get_scratch(freqkv_ctx* ctx, size_t bytes, void** out)
 {
     if (bytes > ctx->scratch_bytes) {
@@ -360,7 +385,8 @@ struct TransformTimer {
 // Compress `count` sequences starting at batch0, all with the same (n_in, n_keep).
 freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, void* v, int32_t batch0,
                              int32_t batch_count, int32_t n_in, int32_t n_keep, int32_t sink, int32_t variant,
-                             cudaStream_t stream, int32_t first = 0)
+                             cudaStream_t stream, int32_t first = 0, GemmState* own_gemm = nullptr,
+                             const Basis* own_basis = nullptr)
 {
     const CacheView view = make_view(l, k, v, batch0, batch_count);
     const int32_t n_mat = 2 * view.mats_per_tensor;
@@ -388,10 +414,16 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
 
     Basis basis;
     const bool gemm = variant == FREQKV_GEMM;
-    freqkv_status st = get_basis(ctx, n_in, n_keep, first, !gemm, gemm, stream, &basis);
+    freqkv_status st = FREQKV_OK;
+    if (own_basis)
+        basis = *own_basis;
+    else
+        st = get_basis(ctx, n_in, n_keep, first, !gemm, gemm, stream, &basis);
     if (st != FREQKV_OK) return st;
 
     if (gemm) {
+        GemmState* gs = own_gemm ? own_gemm : &ctx->gemm;
+        gs->wait_limit_ns = ctx->gemm.wait_limit_ns;
         TransformTimer timer(ctx, stream, false);
         LaunchHooks hooks;
         hooks.user = &timer;
@@ -399,10 +431,10 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
         hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
         const cudaError_t e =
             gemm_is_direct(n_keep)
-                ? launch_gemm_direct(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream)
-                : launch_gemm(&ctx->gemm, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
-        if (e != cudaSuccess) return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm");
-        ctx->kernels_launched += ctx->gemm.kernels_last_call;
+                ? launch_gemm_direct(gs, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream)
+                : launch_gemm(gs, view, basis, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, gs->last_error ? gs->last_error : "launch_gemm");
+        ctx->kernels_launched += gs->kernels_last_call;
         return FREQKV_OK;
     }
 
@@ -745,6 +777,11 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
     WorkOrder order(ctx, stream);  // its end is recorded after the caller's stream has joined the pipeline's tail
     const size_t elt = dtype_size(l.dtype);
     const size_t bytes = (size_t)span_elements(l) * elt;
+    // head stride below one matrix's rows (heads interleaved inside the token axis) is not
+    // something a 2-D copy can express
+    const size_t row_bytes = (size_t)l.stride_token * elt;
+    if (l.kv_heads > 1 && (size_t)l.stride_head * elt < (size_t)(n_in - 1) * row_bytes + (size_t)l.head_dim * elt)
+        return FREQKV_ERR_UNSUPPORTED;
     if (bytes > ctx->stage_bytes) {
         FREQKV_CUDA(ctx, cudaDeviceSynchronize());
         for (int i = 0; i < 2; ++i) {
@@ -756,12 +793,6 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
         FREQKV_CUDA(ctx, cudaMalloc(&ctx->stage[1], bytes));
         ctx->stage_bytes = bytes;
     }
-    // head stride below one matrix's rows (heads interleaved inside the token axis) is not
-    // something a 2-D copy can express
-    const size_t row_bytes = (size_t)l.stride_token * elt;
-    if (l.kv_heads > 1 && (size_t)l.stride_head * elt < (size_t)(n_in - 1) * row_bytes + (size_t)l.head_dim * elt)
-        return FREQKV_ERR_UNSUPPORTED;
-
     // Three-deep pipeline over groups of layers: the host->device copy of group g+1, the
     // compression of group g and the device->host copy of group g-1 run at the same time on three
     // streams of the context (PCIe carries both directions at once), ordered by events; the
@@ -802,31 +833,41 @@ freqkv_status freqkv_compress_host(freqkv_ctx* ctx, const freqkv_layout* layout,
     };
     FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_begin, stream));
     for (int i = 0; i < 3; ++i) FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[i], ctx->pipe_begin, 0));
-    size_t group = 0;
-    for (int32_t b = 0; b < l.batch; ++b)
-        for (int32_t y0 = 0; y0 < l.layers; y0 += per_group, ++group) {
-            const int32_t ny = std::min(per_group, l.layers - y0);
-            cudaEvent_t copied = ctx->pipe_events[2 * group], compressed = ctx->pipe_events[2 * group + 1];
-            cudaError_t e = copy_rows(true, b, y0, ny, sink, n_in, ctx->pipe[0], h2d_bytes);
-            if (e != cudaSuccess) return cuda_fail(ctx, e, "host->device copy");
-            FREQKV_CUDA(ctx, cudaEventRecord(copied, ctx->pipe[0]));
-            FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[1], copied, 0));
-            freqkv_layout sub = l;  // this group's layers of sequence b as a cache of its own
-            sub.batch = 1;
-            sub.layers = ny;
-            const size_t off = ((size_t)b * l.stride_batch + (size_t)y0 * l.stride_layer) * elt;
-            st = compress_group(ctx, sub, static_cast<char*>(ctx->stage[0]) + off, static_cast<char*>(ctx->stage[1]) + off, 0,
-                                1, n_in, kept_len, sink, variant, ctx->pipe[1]);
-            if (st != FREQKV_OK) return st;
-            FREQKV_CUDA(ctx, cudaEventRecord(compressed, ctx->pipe[1]));
-            FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[2], compressed, 0));
-            e = copy_rows(false, b, y0, ny, sink, kept_len, ctx->pipe[2], d2h_bytes);
-            if (e != cudaSuccess) return cuda_fail(ctx, e, "device->host copy");
-        }
-    // every copy back is on pipe[2], after the work it depends on: its tail is the end of the call
-    FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_end, ctx->pipe[2]));
-    FREQKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->pipe_end, 0));
-    return FREQKV_OK;
+    // From here on work may be in flight on the three streams: whatever happens, the caller's
+    // stream joins all of them before this call returns (on an error the host rows are undefined).
+    auto pipeline = [&]() -> freqkv_status {
+        size_t group = 0;
+        for (int32_t b = 0; b < l.batch; ++b)
+            for (int32_t y0 = 0; y0 < l.layers; y0 += per_group, ++group) {
+                const int32_t ny = std::min(per_group, l.layers - y0);
+                cudaEvent_t copied = ctx->pipe_events[2 * group], compressed = ctx->pipe_events[2 * group + 1];
+                cudaError_t e = copy_rows(true, b, y0, ny, sink, n_in, ctx->pipe[0], h2d_bytes);
+                if (e != cudaSuccess) return cuda_fail(ctx, e, "host->device copy");
+                FREQKV_CUDA(ctx, cudaEventRecord(copied, ctx->pipe[0]));
+                FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[1], copied, 0));
+                freqkv_layout sub = l;  // this group's layers of sequence b as a cache of its own
+                sub.batch = 1;
+                sub.layers = ny;
+                const size_t off = ((size_t)b * l.stride_batch + (size_t)y0 * l.stride_layer) * elt;
+                const freqkv_status gs = compress_group(ctx, sub, static_cast<char*>(ctx->stage[0]) + off,
+                                                        static_cast<char*>(ctx->stage[1]) + off, 0, 1, n_in, kept_len, sink,
+                                                        variant, ctx->pipe[1]);
+                if (gs != FREQKV_OK) return gs;
+                FREQKV_CUDA(ctx, cudaEventRecord(compressed, ctx->pipe[1]));
+                FREQKV_CUDA(ctx, cudaStreamWaitEvent(ctx->pipe[2], compressed, 0));
+                e = copy_rows(false, b, y0, ny, sink, kept_len, ctx->pipe[2], d2h_bytes);
+                if (e != cudaSuccess) return cuda_fail(ctx, e, "device->host copy");
+            }
+        return FREQKV_OK;
+    };
+    const freqkv_status run = pipeline();
+    // every copy back is on pipe[2], after the work it depends on; after an error the other two
+    // streams may hold work that nothing on pipe[2] waits for, so all three are joined
+    for (int i = run == FREQKV_OK ? 2 : 0; i < 3; ++i) {
+        FREQKV_CUDA(ctx, cudaEventRecord(ctx->pipe_end, ctx->pipe[i]));
+        FREQKV_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->pipe_end, 0));
+    }
+    return run;
 }
 
 // The context's cos/sin table for `rope_base`, built on `stream` when the base or the capacity has
@@ -971,7 +1012,7 @@ freqkv_status freqkv_attend_prefill(freqkv_ctx* ctx, const freqkv_layout* layout
     {
         TransformTimer timer(ctx, stream);
         e = launch_prefill(l, k, v, layer, q, out, q_heads_per_kv, n_new, lens, table, scale, ctx->prefill_keys,
-                           ctx->prefill_queries, ctx->status_dev, &why, &launched, stream);
+                           ctx->prefill_queries, ctx->status_dev, ctx->gemm.wait_limit_ns, &why, &launched, stream);
     }
     ctx->kernels_launched += launched;
     if (e != cudaSuccess) {
@@ -985,10 +1026,14 @@ freqkv_status freqkv_attend_prefill(freqkv_ctx* ctx, const freqkv_layout* layout
     return FREQKV_OK;
 }
 
+// The graph's kernels have the addresses of the fold scratch and of the basis baked in, so the
+// graph owns both: no later call on the context can free or move them under a replay.
 struct freqkv_decode_graph {
     freqkv_ctx* ctx = nullptr;
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
+    GemmState gemm;
+    Basis basis;
 };
 
 freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, const void* new_k,
@@ -1015,16 +1060,36 @@ freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* l
     // everything that allocates or builds tables happens here, outside the graph
     cudaStream_t cs = nullptr;
     FREQKV_CUDA(ctx, cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
-    Basis basis;
-    st = get_basis(ctx, n_in, kept_len, 0, false, true, cs, &basis);
-    cudaError_t e = st == FREQKV_OK ? cudaStreamSynchronize(cs) : cudaSuccess;
-    if (st == FREQKV_OK && e == cudaSuccess) e = gemm_prepare(&ctx->gemm, gemm_is_direct(kept_len) ? 0 : l.batch * l.layers * l.kv_heads, basis, ctx->sm_count);
     freqkv_decode_graph* dg = new (std::nothrow) freqkv_decode_graph();
+    Basis basis;
+    // a plan of this shape already in the cache may be in use by enqueued kernels and stays there;
+    // the graph gets one of its own, built into the cache and then taken out of it
+    Basis cached;
+    const auto key = std::make_tuple(n_in, kept_len, (int32_t)0);
+    const bool had = ctx->bases.count(key) != 0;
+    if (had) {
+        cached = ctx->bases[key];
+        disown_basis(ctx, n_in, kept_len, 0);
+    }
+    st = dg ? get_basis(ctx, n_in, kept_len, 0, false, true, cs, &basis) : FREQKV_ERR_ALLOC;
+    if (st == FREQKV_OK) {
+        disown_basis(ctx, n_in, kept_len, 0);
+        dg->basis = basis;
+    }
+    if (had) {  // put the context's own plan back
+        ctx->bases[key] = cached;
+        ctx->basis_bytes += basis_device_bytes(cached);
+    }
+    cudaError_t e = st == FREQKV_OK ? cudaStreamSynchronize(cs) : cudaSuccess;
+    if (st == FREQKV_OK && e == cudaSuccess)
+        e = gemm_prepare(&dg->gemm, gemm_is_direct(kept_len) ? 0 : l.batch * l.layers * l.kv_heads, basis, ctx->sm_count);
     auto fail = [&](freqkv_status code, cudaError_t ce, const char* where) {
         if (ce != cudaSuccess) code = cuda_fail(ctx, ce, where);
         if (dg) {
             if (dg->exec) cudaGraphExecDestroy(dg->exec);
             if (dg->graph) cudaGraphDestroy(dg->graph);
+            gemm_release(&dg->gemm);
+            free_basis(&dg->basis);
             delete dg;
         }
         cudaStreamDestroy(cs);
@@ -1058,7 +1123,7 @@ freqkv_status freqkv_decode_graph_create(freqkv_ctx* ctx, const freqkv_layout* l
         ctx->timing = was_timing;
         return fail(FREQKV_ERR_CUDA, e, "capture of the compression");
     }
-    st = compress_group(ctx, l, k, v, 0, l.batch, n_in, kept_len, sink, FREQKV_GEMM, cs);
+    st = compress_group(ctx, l, k, v, 0, l.batch, n_in, kept_len, sink, FREQKV_GEMM, cs, 0, &dg->gemm, &dg->basis);
     e = st == FREQKV_OK ? launch_decode_set_lens(lens_device, l.batch, sink + kept_len, cs) : cudaSuccess;
     cudaGraph_t captured = nullptr;
     const cudaError_t e_end = cudaStreamEndCapture(cs, &captured);
@@ -1082,7 +1147,7 @@ freqkv_status freqkv_decode_graph_launch(freqkv_decode_graph* graph, void* cuda_
     if (!graph || !graph->exec) return FREQKV_ERR_INVALID_ARG;
     DeviceGuard g(graph->ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
-    WorkOrder order(graph->ctx, static_cast<cudaStream_t>(cuda_stream));  // the graph's kernels use the context's scratch
+    WorkOrder order(graph->ctx, static_cast<cudaStream_t>(cuda_stream));  // the graph's kernels use the context's status word
     FREQKV_CUDA(graph->ctx, cudaGraphLaunch(graph->exec, static_cast<cudaStream_t>(cuda_stream)));
     graph->ctx->kernels_launched += 3;  // trigger, append, advance (the compression adds 3 when it runs)
     return FREQKV_OK;
@@ -1095,6 +1160,8 @@ freqkv_status freqkv_decode_graph_destroy(freqkv_decode_graph* graph)
     cudaDeviceSynchronize();
     if (graph->exec) cudaGraphExecDestroy(graph->exec);
     if (graph->graph) cudaGraphDestroy(graph->graph);
+    gemm_release(&graph->gemm);
+    free_basis(&graph->basis);
     cudaGetLastError();
     delete graph;
     return FREQKV_OK;
@@ -1151,6 +1218,24 @@ freqkv_status freqkv_last_device_status(freqkv_ctx* ctx, void* cuda_stream)
         ctx->last_error = buf;
         return FREQKV_ERR_TIMEOUT;
     }
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_set_wait_limit(freqkv_ctx* ctx, int64_t nanoseconds)
+{
+    if (!ctx || nanoseconds < 1000) return FREQKV_ERR_INVALID_ARG;
+    ctx->gemm.wait_limit_ns = (unsigned long long)nanoseconds;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_selftest_bounded_wait(freqkv_ctx* ctx, int64_t nanoseconds, void* cuda_stream)
+{
+    if (!ctx || nanoseconds < 1000 || nanoseconds > 1000000000ll) return FREQKV_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return FREQKV_ERR_CUDA;
+    const cudaError_t e = launch_wait_probe(ctx->status_dev, (unsigned long long)nanoseconds, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bounded wait probe");
+    ctx->kernels_launched += 1;
     return FREQKV_OK;
 }
 

@@ -656,16 +656,17 @@ __global__ void rope_table_kernel(float2* table, int32_t rows, double base)
 
 cudaError_t launch_mma(const AttendParams& prm, int32_t g, int32_t nb, cudaStream_t stream)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attrs;
+    const cudaError_t attr_error = attrs.run([] {
         const void* kernels[3] = {(const void*)attend_mma_kernel<2>, (const void*)attend_mma_kernel<4>, (const void*)attend_mma_kernel<8>};
         for (const void* f : kernels) {
             cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, MMA_SMEM_BYTES);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             if (e != cudaSuccess) return e;
         }
-        attr_set = true;
-    }
+        return cudaSuccess;
+    });
+    if (attr_error != cudaSuccess) return attr_error;
     const dim3 grid((unsigned)prm.splits, (unsigned)(nb * prm.kv_heads));
     switch (g) {
         case 2: attend_mma_kernel<2><<<grid, MMA_THREADS, MMA_SMEM_BYTES, stream>>>(prm); break;

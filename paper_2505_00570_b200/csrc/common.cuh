@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "freqkv.h"
 
 namespace freqkv {
@@ -82,6 +84,26 @@ cudaError_t launch_decode_set_lens(int32_t* lens, int32_t batch, int32_t value, 
 // rows at lens[b] <- the new rows ([batch, layers, kv_heads, 1, head_dim]), then lens[b] += 1 (full sequences skipped)
 cudaError_t launch_decode_append(const CacheView& view, int32_t dtype, int32_t batch, int32_t* lens, int32_t capacity,
                                  const void* new_k, const void* new_v, cudaStream_t stream);
+
+// Set-up that must run once per DEVICE (cudaFuncSetAttribute applies to the current device only):
+// run(f) calls f() the first time it is reached with a given device current, under a mutex.
+struct PerDeviceOnce {
+    std::mutex mutex;
+    bool done[64] = {};
+    template <class F>
+    cudaError_t run(F&& f)
+    {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        std::lock_guard<std::mutex> lock(mutex);
+        if (dev < 0 || dev >= 64) return f();
+        if (done[dev]) return cudaSuccess;
+        e = f();
+        if (e == cudaSuccess) done[dev] = true;
+        return e;
+    }
+};
 
 inline size_t dtype_size(int32_t dtype) { return dtype == FREQKV_F32 ? 4 : 2; }
 

@@ -454,18 +454,16 @@ void fdct_free_plan(FdctPlan* plan)
 cudaError_t launch_fdct(const CacheView& view, int32_t dtype, int32_t n_mat, const FdctPlan& plan, int32_t sink,
                         cudaStream_t stream)
 {
-    static bool attr_set[2] = {false, false};
+    static PerDeviceOnce attrs;
     const size_t smem = smem_bytes(plan.n_in);
-    if (!attr_set[dtype == FREQKV_F32]) {
+    const cudaError_t attr_error = attrs.run([] {
         const size_t max_smem = smem_bytes(128);  // the largest footprint (most pairs, most padding rows)
-        const cudaError_t e =
-            dtype == FREQKV_F32
-                ? cudaFuncSetAttribute(fdct_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem)
-                : cudaFuncSetAttribute(fdct_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)max_smem);
-        if (e != cudaSuccess) return e;
-        attr_set[dtype == FREQKV_F32] = true;
-    }
+        cudaError_t e = cudaFuncSetAttribute(fdct_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(fdct_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        return e;
+    });
+    if (attr_error != cudaSuccess) return attr_error;
     FdctParams prm;
     prm.log_n = ilog2(plan.n_in);
     prm.log_l = ilog2(plan.n_keep);

@@ -11,6 +11,7 @@ struct GemmState {
     int max_clusters = 0;     // CTA pairs that can be resident at once
     void* scratch = nullptr;  // folded inputs U, V: [pairs][K|V][U|V][ceil(n_in/2)][128] bf16 per pass
     size_t scratch_bytes = 0;
+    unsigned long long wait_limit_ns = 2000000000ull;  // bound of every mbarrier wait inside the kernel (2 s)
 };
 
 // Called on the launching stream right before and right after the tensor-core kernel itself
@@ -38,5 +39,8 @@ bool gemm_is_direct(int32_t n_keep);
 cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
                                int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 void gemm_release(GemmState* state);
+// A one-thread kernel that waits, with the tensor-core kernel's own bounded wait, on an mbarrier
+// nothing arrives on: after `limit_ns` it sets a bit in *status_dev and returns.
+cudaError_t launch_wait_probe(int32_t* status_dev, unsigned long long limit_ns, cudaStream_t stream);
 
 }  // namespace freqkv

@@ -1,9 +1,8 @@
 // freqkv_compress_noalloc: the CUDA-core compression for callers that must not allocate.
 //
-// Some callers cannot call cudaMalloc at all: code running between the begin and end of a CUDA
-// stream capture (allocation is not a capturable operation), code holding a lock that the
-// allocator's implicit device synchronisation would deadlock against, real-time serving loops
-// with a frozen memory budget, and plug-ins whose host framework owns every byte of device memory.
+// Some callers cannot call cudaMalloc at all: code holding a lock that the allocator's implicit
+// device synchronisation would deadlock against, real-time serving loops with a frozen memory
+// budget, and plug-ins whose host framework owns every byte of device memory.
 // freqkv_compress needs a context (freqkv_create allocates) plus a plan and an output staging
 // buffer obtained from cudaMalloc on first use.  This entry point needs none of that: the
 // projection basis and the output staging live in two file-scope __device__ arrays of fixed
@@ -79,9 +78,12 @@ extern "C" freqkv_status freqkv_compress_noalloc(const freqkv_layout* layout, vo
     const size_t per_matrix = (size_t)kept_len * layout->head_dim * dtype_size(layout->dtype);
     if (per_matrix > kStagingBytes) return FREQKV_ERR_UNSUPPORTED;
 
-    // The arrays used are those of the device that owns the cache.
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, k) != cudaSuccess || attr.type != cudaMemoryTypeDevice) {
+    // The arrays used are those of the device that owns the cache: K and V must be plain device
+    // memory of one and the same device.
+    cudaPointerAttributes attr, attr_v;
+    if (cudaPointerGetAttributes(&attr, k) != cudaSuccess || attr.type != cudaMemoryTypeDevice ||
+        cudaPointerGetAttributes(&attr_v, v) != cudaSuccess || attr_v.type != cudaMemoryTypeDevice ||
+        attr_v.device != attr.device) {
         cudaGetLastError();
         return FREQKV_ERR_INVALID_ARG;
     }

@@ -59,7 +59,6 @@ constexpr int SMEM_BYTES = SMEM_USED + 1024;  // + slack for aligning the base t
 static_assert(2 * (SMEM_BYTES + 1024) <= 233472, "two CTAs per SM (1 KB of each CTA's share is reserved)");
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 256;      // S buffers in columns 0..63 and 64..127, O in 128..255
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 constexpr unsigned long long LANDING_NS = 1000000ull;        // 1 ms
 constexpr float NEG_INF = -INFINITY;
 constexpr float RESCALE_STEP = 8.f;  // log2 of the largest weight the lazy reference allows
@@ -68,6 +67,7 @@ struct PrefillParams {
     int32_t n_new, kv_heads, g, layer, batch0, batch_count, q_tiles;
     __nv_bfloat16* out;  // [batch, kv_heads * g, n_new, 128]
     int32_t* status;
+    unsigned long long wait_limit_ns;  // bound of every mbarrier wait
     int32_t len[PREFILL_MAX_BATCH];
 };
 
@@ -109,8 +109,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Wait for the phase with the given parity.  Gives up when another role has raised the abort flag
-// or after WAIT_LIMIT_NS (then it sets the status bit and raises the flag).  False = gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+// or after `limit_ns` (then it sets the status bit and raises the flag).  False = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
@@ -118,7 +119,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (global_timer_ns() - t0 > limit_ns) {
             atomicOr(status, PREFILL_ERR_WAIT);
             *abort_flag = 1;
             __threadfence_block();
@@ -372,11 +373,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             tma_load_3d(base + OFF_Q + Q_SLAB, &map_q, q_full, 64, q0, q_slice);
             for (int32_t t = 0; t < n_tiles; ++t) {
                 const int sk = t % RING_K, sv = t % RING_V;
-                if (t >= RING_K && !mbar_wait(k_empty(sk), ((uint32_t)(t / RING_K) - 1) & 1, abort_flag, prm.status)) break;
+                if (t >= RING_K && !mbar_wait(k_empty(sk), ((uint32_t)(t / RING_K) - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) break;
                 mbar_expect_tx(k_full(sk), KV_TILE);
                 tma_load_3d(base + OFF_K + sk * KV_TILE, &map_k, k_full(sk), 0, t * BKV, k_slice);
                 tma_load_3d(base + OFF_K + sk * KV_TILE + KV_SLAB, &map_k, k_full(sk), 64, t * BKV, k_slice);
-                if (t >= RING_V && !mbar_wait(v_empty(sv), ((uint32_t)(t / RING_V) - 1) & 1, abort_flag, prm.status)) break;
+                if (t >= RING_V && !mbar_wait(v_empty(sv), ((uint32_t)(t / RING_V) - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) break;
                 mbar_expect_tx(v_full(sv), KV_TILE);
                 tma_load_5d(base + OFF_V + sv * KV_TILE, &map_v, v_full(sv), 0, t * BKV, h, prm.layer, prm.batch0 + b);
                 tma_load_5d(base + OFF_V + sv * KV_TILE + KV_SLAB, &map_v, v_full(sv), 64, t * BKV, h, prm.layer, prm.batch0 + b);
@@ -389,11 +390,11 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            bool alive = mbar_wait(q_full, 0, abort_flag, prm.status);
+            bool alive = mbar_wait(q_full, 0, abort_flag, prm.status, prm.wait_limit_ns);
             auto issue_scores = [&](int32_t t) {
                 const int s = t % RING_K;
-                if (!mbar_wait(k_full(s), (uint32_t)(t / RING_K) & 1, abort_flag, prm.status)) return false;
-                if (t >= 2 && !mbar_wait(s_free(t & 1), ((uint32_t)(t / 2) - 1) & 1, abort_flag, prm.status)) return false;
+                if (!mbar_wait(k_full(s), (uint32_t)(t / RING_K) & 1, abort_flag, prm.status, prm.wait_limit_ns)) return false;
+                if (t >= 2 && !mbar_wait(s_free(t & 1), ((uint32_t)(t / 2) - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t qa = base + OFF_Q, ka = base + OFF_K + s * KV_TILE;
 #pragma unroll
@@ -408,8 +409,8 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             for (int32_t t = 0; t < n_tiles && alive; ++t) {
                 if (t + 1 < n_tiles && !issue_scores(t + 1)) break;
                 const int s = t % RING_V;
-                if (!mbar_wait(p_ready, t & 1, abort_flag, prm.status)) break;
-                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status)) break;
+                if (!mbar_wait(p_ready, t & 1, abort_flag, prm.status, prm.wait_limit_ns)) break;
+                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status, prm.wait_limit_ns)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t va = base + OFF_V + s * KV_TILE;
 #pragma unroll
@@ -432,7 +433,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         for (int32_t t = 0; t < n_tiles; ++t) {
             const int buf = t & 1, s = t % RING_V;
             const int32_t j0 = t * BKV;
-            if (!mbar_wait(s_full(buf), (t / 2) & 1, abort_flag, prm.status)) { alive = false; break; }
+            if (!mbar_wait(s_full(buf), (t / 2) & 1, abort_flag, prm.status, prm.wait_limit_ns)) { alive = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             uint32_t sc[64];
             tmem_ld32<0>(tmem_base + lane_bits + buf * BKV + 0, sc);
@@ -470,7 +471,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             l_run += (s4[0] + s4[1]) + (s4[2] + s4[3]);
 
             if (t > 0) {  // the previous tile's P V must have finished: P is free, O is at rest
-                if (!mbar_wait(o_full, (t - 1) & 1, abort_flag, prm.status)) { alive = false; break; }
+                if (!mbar_wait(o_full, (t - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) { alive = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
@@ -492,7 +493,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (j0 + BKV > len) {  // value rows past the cache length are stale: make them zeros
-                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status)) { alive = false; break; }
+                if (!mbar_wait(v_full(s), (uint32_t)(t / RING_V) & 1, abort_flag, prm.status, prm.wait_limit_ns)) { alive = false; break; }
                 if (row < BKV && j0 + row >= len) {
                     uint8_t* v_row = aligned + OFF_V + s * KV_TILE + row * 128;
 #pragma unroll
@@ -505,7 +506,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             }
             mbar_arrive(p_ready);
         }
-        if (alive && mbar_wait(o_full, (n_tiles - 1) & 1, abort_flag, prm.status)) {
+        if (alive && mbar_wait(o_full, (n_tiles - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const float inv = 1.f / l_run;
             const bool store = q0 + row < prm.n_new;
@@ -598,22 +599,22 @@ size_t prefill_query_scratch_bytes(const freqkv_layout& l, int32_t q_heads_per_k
 
 cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v, int32_t layer, const void* q, void* out,
                            int32_t g, int32_t n_new, const int32_t* lens_host, const float2* table, float scale,
-                           void* key_scratch, void* query_scratch, int32_t* status, const char** error,
-                           int32_t* kernels_launched, cudaStream_t stream)
+                           void* key_scratch, void* query_scratch, int32_t* status, unsigned long long wait_limit_ns,
+                           const char** error, int32_t* kernels_launched, cudaStream_t stream)
 {
     *error = nullptr;
     if (!encode_fn()) {
         *error = "cuTensorMapEncodeTiled is not available from this driver";
         return cudaErrorNotSupported;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attrs;
+    const cudaError_t attr_error = attrs.run([] {
         cudaError_t e = cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+        return e;
+    });
+    if (attr_error != cudaSuccess) return attr_error;
     const int32_t heads_q = l.kv_heads * g;
     CUtensorMap map_q, map_k, map_v;
     if (!encode_rows_map(&map_q, query_scratch, n_new, (int64_t)l.batch * heads_q, BQ) ||
@@ -661,6 +662,7 @@ cudaError_t launch_prefill(const freqkv_layout& l, const void* k, const void* v,
         prm.q_tiles = (n_new + BQ - 1) / BQ;
         prm.out = static_cast<__nv_bfloat16*>(out);
         prm.status = status;
+        prm.wait_limit_ns = wait_limit_ns;
         const dim3 grid((unsigned)((int64_t)prm.q_tiles * heads_q * nb));
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = grid;

@@ -92,16 +92,37 @@ def ar1_rows(
     pass ``state`` back in to continue the same sequences (None starts them).
     """
     b = w.batch if batch is None else batch
-    shape = (b, w.layers, w.kv_heads, w.head_dim)
+    cols = b * w.layers * w.kv_heads * w.head_dim
     out = torch.empty((b, w.layers, w.kv_heads, n_tokens, w.head_dim), dtype=w.dtype, device=device)
     innov = (1.0 - w.rho * w.rho) ** 0.5
-    block = 256
-    for n0 in range(0, n_tokens, block):
+    # The recursion runs a block of tokens at a time as one matrix product: inside a block
+    #   x_j = rho^(j+1) * x_prev + innov * sum_{i <= j} rho^(j-i) * e_i
+    # (a lower-triangular Toeplitz matrix applied to the block's innovations), so a block costs
+    # a handful of launches instead of a few per token.  Block size bounded by memory.
+    block = max(16, min(1024, (1 << 28) // max(cols, 1)))
+    steps = torch.arange(block, device=device, dtype=torch.float64)
+    lag = steps[:, None] - steps[None, :]
+    toeplitz = torch.where(lag >= 0, innov * torch.pow(torch.tensor(w.rho, dtype=torch.float64, device=device), lag.clamp(min=0)),
+                           torch.zeros((), dtype=torch.float64, device=device)).to(torch.float32)
+    carry = torch.pow(torch.tensor(w.rho, dtype=torch.float64, device=device), steps + 1).to(torch.float32)
+    n0 = 0
+    while n0 < n_tokens:
         nb = min(block, n_tokens - n0)
-        eps = torch.randn((nb,) + shape, generator=gen, device=device, dtype=torch.float32)
-        for j in range(nb):
-            state = eps[j] if state is None else w.rho * state + innov * eps[j]
-            out[:, :, :, n0 + j, :] = (state * scales).to(w.dtype)
+        eps = torch.randn((nb, cols), generator=gen, device=device, dtype=torch.float32)
+        if state is None:
+            # the very first token is the stationary draw itself: x_0 = e_0
+            state = eps[0].clone()
+            x = torch.empty_like(eps)
+            x[0] = state
+            if nb > 1:
+                x[1:] = toeplitz[:nb - 1, :nb - 1] @ eps[1:] + carry[:nb - 1, None] * state[None, :]
+        else:
+            x = toeplitz[:nb, :nb] @ eps + carry[:nb, None] * state.reshape(-1)[None, :]
+        state = x[nb - 1].clone()
+        scaled = x.view(nb, b, w.layers, w.kv_heads, w.head_dim) * scales
+        out[:, :, :, n0:n0 + nb, :] = scaled.permute(1, 2, 3, 0, 4).to(w.dtype)
+        n0 += nb
+    state = state.view(b, w.layers, w.kv_heads, w.head_dim)
     return out, state
 
 

@@ -306,6 +306,25 @@ def test_band_config2_shape_high_frequencies(ctx):
     parity.check_compress(ctx, w, 4096, 2046, 4, fk.AUTO, sample=4, first=2046)
 
 
+@pytest.mark.parametrize("variant,dtype", [(fk.GEMM, torch.bfloat16), (fk.SIMT, torch.bfloat16), (fk.SIMT, torch.float32)])
+@pytest.mark.parametrize("rho", [-0.9, 0.0])
+@pytest.mark.parametrize("n_in,kept,first", [(300, 150, 150), (301, 150, 151), (1024, 512, 512), (1000, 333, 667), (700, 300, 201)])
+def test_band_with_energy_in_the_band_plain_metric(ctx, variant, dtype, rho, n_in, kept, first):
+    """Retaining High/Low-Frequency Components (the paper's ablation) on inputs that HAVE energy in
+    the retained band -- an AR(1) process with rho = -0.9 (energy at the high frequencies) and white
+    noise (rho = 0) -- held to the plain metric |Y_gpu - Y_oracle| / |Y_oracle| <= 1e-2 (bf16),
+    1e-5 (fp32); even and odd first components (opposite signs in the tensor-core epilogue)."""
+    w = small(cap=n_in + 7, dtype=dtype, sink=4, rho=rho, outliers=2 if dtype == torch.bfloat16 else 0, Ly=2, H=2)
+    parity.check_compress(ctx, w, n_in + 4, kept, 4, variant, first=first, band_plain=True)
+
+
+@pytest.mark.parametrize("rho", [-0.9, 0.0])
+def test_band_config2_shape_high_frequencies_plain_metric(ctx, rho):
+    """The highest 2046 of 4092 components on the 7B shape, input energy in that band, plain metric."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2_7b"], layers=1, kv_heads=4, rho=rho)
+    parity.check_compress(ctx, w, 4096, 2046, 4, fk.AUTO, sample=8, first=2046, band_plain=True)
+
+
 def test_band_invalid_and_fast_transform(ctx):
     k = torch.zeros(1, 1, 1, 600, 128, device="cuda", dtype=torch.bfloat16)
     v = torch.zeros_like(k)

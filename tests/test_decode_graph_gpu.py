@@ -62,6 +62,55 @@ def test_decode_graph_equals_host_driven_stream(ctx, cap, sink, kept, T):
         graph.close()
 
 
+def test_decode_graph_survives_larger_calls_on_its_context(ctx):
+    """The graph's kernels have the addresses of the fold scratch and of the basis baked in.  Other
+    calls on the same context that need a larger scratch (a bigger cache) or rebuild plans must not
+    move or free what a live graph replays from: the graph owns its own.  The stream through the
+    graph, with such calls in between, must still be bit-identical to the host-driven one."""
+    cap, sink, kept, T = 300, 4, 148, 700
+    w = synth.Workload("dg", 2, 2, 2, 128, cap, torch.bfloat16, sink, 0.9, 2, synth.BASE_SEED + 43)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    scales = synth.channel_scales(w, gen, "cuda")
+    toks, _ = synth.ar1_rows(w, T, gen, "cuda", scales)
+    big = synth.Workload("dg_big", 3, 4, 4, 128, 1500, torch.bfloat16, sink, 0.9, 2, synth.BASE_SEED + 44)
+    ctx.set_variant(fk.GEMM)
+    k1, v1 = synth.make_cache(w, "cuda", fill_len=0)
+    lens = [0, 0]
+    for t in range(T):
+        nk = toks[:, :, :, t:t + 1].contiguous()
+        try:
+            lens = ctx.append(k1, v1, nk, nk, lens)
+        except fk.FreqKVError as e:
+            assert e.status == fk.ERR_CAPACITY
+            n = ctx.compress(k1, v1, cap, kept, sink)
+            lens = ctx.append(k1, v1, nk, nk, [n, n])
+    k2, v2 = synth.make_cache(w, "cuda", fill_len=0)
+    lens_dev = torch.zeros(2, dtype=torch.int32, device="cuda")
+    stage_k = torch.empty_like(toks[:, :, :, :1]).contiguous()
+    stage_v = torch.empty_like(stage_k)
+    graph = fk.DecodeGraph(ctx, k2, v2, stage_k, stage_v, lens_dev, kept, sink)
+    try:
+        for t in range(T):
+            if t in (10, 350):   # a call that needs a much larger fold scratch, and the graph's own shape again
+                kb, vb = synth.make_cache(big, "cuda")
+                ctx.compress(kb, vb, 1500, 748, sink)
+                ks, vs = synth.make_cache(w, "cuda")
+                ctx.compress(ks, vs, cap, kept, sink)
+                del kb, vb, ks, vs
+            stage_k.copy_(toks[:, :, :, t:t + 1])
+            stage_v.copy_(toks[:, :, :, t:t + 1])
+            graph.launch()
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == fk.OK
+        assert lens_dev.tolist() == lens
+        n = lens[0]
+        assert torch.equal(k2[:, :, :, :n], k1[:, :, :, :n]) and torch.equal(v2[:, :, :, :n], v1[:, :, :, :n])
+    finally:
+        graph.close()
+        ctx.set_variant(fk.AUTO)
+
+
 def test_decode_graph_reports_a_batch_that_is_not_uniform(ctx):
     w = synth.Workload("dg", 2, 1, 1, 128, 200, torch.bfloat16, 4, 0.9, 0, synth.BASE_SEED + 42)
     k, v = synth.make_cache(w, "cuda")

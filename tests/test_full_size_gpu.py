@@ -64,26 +64,28 @@ def check_uniform(ctx, name: str, sample: int):
     for t, hd, tl in zip((k, v), head, tail):
         assert torch.equal(t[..., :sink, :], hd), "sink rows changed"
         assert torch.equal(t[..., sink + kept:, :], tl), "rows past the new length changed"
-    worst = 0.0
+    assert len(ids) >= min(32, w.n_matrices) and ids[0] == 0 and ids[-1] == w.n_matrices - 1
+    worst = worst_row = worst_channel = 0.0
     for i in ids:
         t, b, l, h = coords(i, k.shape)
         want = oracle.compress_matrix(inputs[i], kept)
         got = parity.to_f64((k, v)[t][b, l, h, sink:sink + kept])
-        worst = max(worst, parity.rel_l2(got, want))
-    assert worst <= TOL_BF16, f"{name}: relative L2 {worst:.3e}"
+        m, r, c = parity.check_matrix(got, want, torch.bfloat16, f"{name} matrix {i}")
+        worst, worst_row, worst_channel = max(worst, m), max(worst_row, r), max(worst_channel, c)
+    print(f"{name}: {len(ids)} matrices, worst matrix {worst:.3e}, worst row {worst_row:.3e}, worst channel {worst_channel:.3e}")
     return worst
 
 
 def test_config2_llama2_7b_full(ctx):
     """32 x 32 heads x 128, 4096 tokens, 4 sinks, 4092 -> 2046: 2048 matrices in one call."""
     need_gib(20)
-    check_uniform(ctx, "llama2_7b", sample=24)
+    check_uniform(ctx, "llama2_7b", sample=32)
 
 
 def test_config3_llama3_8b_full(ctx):
     """Batch 8, 32 x 8 KV heads x 128, 8192 tokens, 8188 -> 4094: 4096 matrices in one call."""
     need_gib(40)
-    check_uniform(ctx, "llama3_8b", sample=10)
+    check_uniform(ctx, "llama3_8b", sample=32)
 
 
 def test_config5b_ragged_full(ctx):
@@ -105,15 +107,22 @@ def test_config5b_ragged_full(ctx):
             assert torch.equal(t_out[b, :, :, sink + kept[b]:], t_in[b, :, :, sink + kept[b]:])
     gen = torch.Generator().manual_seed(w.seed + 9)
     seqs = {min(range(w.batch), key=lambda b: lens[b]), max(range(w.batch), key=lambda b: lens[b]), 0, w.batch - 1}
-    seqs |= set(torch.randperm(w.batch, generator=gen)[:3].tolist())
-    worst = 0.0
+    for b in torch.randperm(w.batch, generator=gen).tolist():
+        if len(seqs) >= 8:
+            break
+        seqs.add(b)
+    worst = worst_row = 0.0
+    checked = 0
     for b in sorted(seqs):
         for (l, h) in ((0, 0), (w.layers - 1, w.kv_heads - 1)):
             for t_in, t_out in ((k_in, k), (v_in, v)):
                 want = oracle.compress_matrix(parity.to_f64(t_in[b, l, h, sink:lens[b]]), kept[b])
                 got = parity.to_f64(t_out[b, l, h, sink:sink + kept[b]])
-                worst = max(worst, parity.rel_l2(got, want))
-    assert worst <= TOL_BF16, f"ragged: relative L2 {worst:.3e}"
+                m, r, _ = parity.check_matrix(got, want, torch.bfloat16, f"ragged sequence {b} (length {lens[b]})")
+                worst, worst_row = max(worst, m), max(worst_row, r)
+                checked += 1
+    assert checked >= 32
+    print(f"ragged: {checked} matrices, worst matrix {worst:.3e}, worst row {worst_row:.3e}")
 
 
 def test_config4_decode_stream_full(ctx):
@@ -124,7 +133,7 @@ def test_config4_decode_stream_full(ctx):
     cap, sink, total = w.capacity, w.sink, 32768
     kept = w.kept_len(cap)
     k, v = synth.make_cache(w, "cuda", fill_len=0)
-    ids = synth.sample_matrix_ids(w.n_matrices, 4, w.seed + 5)
+    ids = synth.sample_matrix_ids(w.n_matrices, 8, w.seed + 5)
     where = [coords(i, k.shape) for i in ids]
     gens, scales, state = [], [], [None, None]
     for which in range(2):
@@ -170,7 +179,7 @@ def test_config5a_chunked_prefill_full(ctx):
     cap, sink, total, chunk = w.capacity, w.sink, 262144, 4096
     kept = w.kept_len(cap)
     k, v = synth.make_cache(w, "cuda", fill_len=0)
-    ids = [0, w.n_matrices - 1]
+    ids = synth.sample_matrix_ids(w.n_matrices, 8, w.seed + 5)
     where = [coords(i, k.shape) for i in ids]
     gens, scales, state = [], [], [None, None]
     for which in range(2):

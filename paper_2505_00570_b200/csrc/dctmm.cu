@@ -1,0 +1,777 @@
+// Fast transform on the tensor cores.
+//
+// The compression of one channel (Section 3.3, Eq. 2-3: DCT-II of N rows, keep L components,
+// L-point inverse, rescale by sqrt(L/N)) is computed the way Appendix A points to -- "the DCT can
+// be computed using the FFT", O(N log N) instead of the O(L N) of a dense projection -- with the
+// FFT's factors executed as small dense matrix products on the tcgen05 tensor cores:
+//
+//   forward, N = N1 N2     v = reordered input (v_p = x_2p, v_{N-1-p} = x_{2p+1}),  p = N2 n1 + n2
+//     stage 1  (over n1)   A[t1, n2] = sum_n1 exp(-2 pi i n1 t1 / N1) v[n1, n2],   t1 <= N1/2 (real input:
+//                          the other half is the conjugate)
+//     twiddle              A~ = A * exp(-i pi t1 (4 n2 + 1) / (2N))          (CUDA cores, fp32)
+//     stage 2  (over n2)   U_t = exp(-i pi t2 / (2 N2)) sum_n2 exp(-2 pi i n2 t2 / N2) A~[t1, n2],  t = t1 + N1 t2;
+//                          the DCT components are  z_t = Re U_t  and  z_{N-t} = -Im U_t
+//   keep t < L; all normalisations (orthonormal DCT and inverse, sqrt(L/N)) multiply to 2/N
+//   inverse, L = L1 L2     r = Re IDFT_L(h_t exp(i pi t / (2L))) in Hermitian form, t = t1 + L1 t2, j = L2 j1 + j2
+//     stage 3  (over t2)   C[t1, j2] = sum_t2 g[j2, t2] (h_{t1 + L1 t2} - i h_{L - t1 - L1 t2}),  t1 <= L1/2,
+//                          g = exp(i pi t2 / (2 L2)) exp(2 pi i j2 t2 / L2) / 2
+//     twiddle              C~ = C * exp(i pi t1 (4 j2 + 1) / (2L))
+//     stage 4  (over t1)   r[j1, j2] = sum_t1 w_t1 Re(exp(2 pi i j1 t1 / L1) C~[t1, j2]),  y_{2j} = r_j, y_{2j+1} = r_{L-1-j}
+//
+// Each stage is D = F B with F a real matrix of at most 128 rows (the real and imaginary parts of
+// a complex stage are separate rows) and B the data: contraction index down the rows, (outer
+// index, channel) along the columns.  Work is cut into slabs of one matrix x 8 channels (one
+// 16-byte piece of every row): a slab's N x 8 values stay in shared memory through all four
+// stages and its L output rows are written over its own input rows, so the transform is in place
+// in global memory with no scratch -- no other CTA touches those channels.
+//
+// One persistent CTA per SM:
+//   warps 0-7   load the slab (cp.async, each 16-byte piece placed where stage 1 wants it), and
+//               after every stage move the accumulators from tensor memory to the next stage's
+//               operand in shared memory (twiddle, round to bf16, re-index) or, after stage 4, to
+//               the cache; warp w works on TMEM lanes 32 (w % 4) .. +31 and on every second
+//               64-column group;
+//   warp 8      issues the tcgen05.mma instructions (M 128, N up to 256, K 16; bf16 in, fp32 out)
+//               of one 256-column chunk at a time into one of two halves of tensor memory, so
+//               that the products of a chunk overlap the movement of the previous one.
+// The four matrices F stay resident in shared memory (copied once per CTA from a pre-swizzled
+// image).  Two data buffers alternate between stages; the next slab's load starts as soon as
+// stage 3 has consumed the buffer it goes to.  Every barrier wait is bounded in time.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
+#include "dctmm.cuh"
+
+namespace freqkv {
+namespace {
+
+constexpr int EPI_WARPS = 8;
+constexpr int EPI_THREADS = EPI_WARPS * 32;
+constexpr int THREADS = EPI_THREADS + 32;
+constexpr int CHUNK_ATOMS = 4;                 // 4 x 64 columns = N 256 per instruction
+constexpr int TMEM_COLS = 512;
+constexpr int SMEM_LIMIT = 232448 - 1024;      // opt-in maximum minus alignment slack
+constexpr int MAX_N = 8192;
+
+struct DctmmParams {
+    DctmmPlan plan;
+    int32_t sink, slabs_per_matrix, total_slabs;
+    float inv_n2, inv_l1;
+    int32_t* status;
+    unsigned long long wait_limit_ns;
+};
+
+// ---------------------------------------------------------------------------------- device helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Wait for the phase with the given parity; gives up when another thread has raised the abort
+// flag or after limit_ns (then it sets the status bit and raises the flag).  False = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          unsigned long long limit_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > limit_ns) {
+            atomicOr(status, DCTMM_ERR_WAIT);
+            *abort_flag = 1;
+            __threadfence_block();
+            return false;
+        }
+    }
+}
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading and stride byte offsets
+// (16-byte units), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, A K-major, B MN-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t idesc_for(uint32_t n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive columns of tensor memory into registers.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32])
+{
+    uint32_t u[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
+          "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
+          "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ uint4 pack8(const float* v)
+{
+    return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+__device__ __forceinline__ void st_shared_16(uint32_t addr, const uint4& v)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// Byte offset, inside a stage's B buffer, of the 16-byte piece (contraction index k, outer index o):
+// 64-column groups ("atoms", 8 outer values x 8 channels) are k_pad rows of 128 bytes each; the
+// eight pieces of a row are permuted by the row number (128-byte swizzle).
+__host__ __device__ __forceinline__ uint32_t b_piece(uint32_t k, uint32_t o, uint32_t k_pad)
+{
+    return (o >> 3) * (k_pad * 128u) + k * 128u + (((o & 7u) ^ (k & 7u)) << 4);
+}
+
+// q = t / d, r = t % d for 0 <= t < 2^15, 1 <= d <= 2^8 through one multiplication (exact: the
+// half added to t keeps the product at least 0.5 / d away from an integer, far more than the
+// rounding of a float product of this size).
+__device__ __forceinline__ void divmod_small(int32_t t, int32_t d, float inv_d, int32_t* q, int32_t* r)
+{
+    *q = (int32_t)(((float)t + 0.5f) * inv_d);
+    *r = t - *q * d;
+}
+
+// cos and sin of pi * num / den for integers 0 <= num < 2 den.
+__device__ __forceinline__ void sincos_ratio(int32_t num, int32_t den, float* s, float* c)
+{
+    sincospif((float)num / (float)den, s, c);
+}
+
+// ---------------------------------------------------------------------------------- the kernel
+
+__global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheView view, const DctmmParams prm)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const DctmmPlan& P = prm.plan;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* aligned = smem_raw + (base - raw);
+    // barriers: ready[0..3] (stage s operand complete), acc_full[0..1], acc_empty[0..1]
+    const uint32_t bar0 = base + P.bar_off;
+    auto ready_bar = [&](int s) { return bar0 + 8u * s; };
+    auto full_bar = [&](int b) { return bar0 + 8u * (4 + b); };
+    auto empty_bar = [&](int b) { return bar0 + 8u * (6 + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aligned + P.bar_off + 64);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int32_t* status = prm.status;
+    (void)status;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 4; ++s) mbar_init(ready_bar(s), EPI_THREADS);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(full_bar(b), 1);
+            mbar_init(empty_bar(b), EPI_WARPS);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == EPI_WARPS) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    // the matrices F: a plain copy of the pre-swizzled image; both data buffers start as zeros
+    // (never-written padding must not hold NaN bit patterns: it meets zero entries of F)
+    {
+        const uint4* img = static_cast<const uint4*>(P.image);
+        uint4* dst = reinterpret_cast<uint4*>(aligned);
+        const int32_t n_f = P.f_bytes / 16, n_all = P.bar_off / 16;
+        for (int32_t i = threadIdx.x; i < n_f; i += THREADS) dst[i] = img[i];
+        for (int32_t i = n_f + threadIdx.x; i < n_all; i += THREADS) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int32_t n_iter = prm.total_slabs > (int32_t)blockIdx.x
+                               ? (prm.total_slabs - (int32_t)blockIdx.x + (int32_t)gridDim.x - 1) / (int32_t)gridDim.x
+                               : 0;
+
+    if (warp == EPI_WARPS) {
+        // ------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            uint32_t q = 0;  // chunk counter: tensor-memory half q & 1
+            bool alive = true;
+            for (int32_t it = 0; it < n_iter && alive; ++it) {
+                for (int s = 0; s < 4 && alive; ++s) {
+                    const DctmmStage& st = P.st[s];
+                    if (!mbar_wait(ready_bar(s), it & 1, abort_flag, prm.status, prm.wait_limit_ns)) {
+                        alive = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_base = base + st.a_off, b_base = base + st.b_off;
+                    const uint32_t tile_bytes = (uint32_t)st.rows8 * 128u, lbo = (uint32_t)st.k_pad * 128u;
+                    const int32_t k_steps = st.k_pad / 16;
+                    for (int32_t a0 = 0; a0 < st.atoms; a0 += CHUNK_ATOMS, ++q) {
+                        const uint32_t buf = q & 1u;
+                        if (q >= 2 && !mbar_wait(empty_bar(buf), ((q >> 1) - 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) {
+                            alive = false;
+                            break;
+                        }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t n_atoms = (uint32_t)min(CHUNK_ATOMS, st.atoms - a0);
+                        const uint32_t idesc = idesc_for(64u * n_atoms);
+                        for (int32_t ks = 0; ks < k_steps; ++ks) {
+                            const uint64_t ad = smem_desc(a_base + (uint32_t)(ks >> 2) * tile_bytes + (uint32_t)(ks & 3) * 32u, 16, 1024);
+                            const uint64_t bd = smem_desc(b_base + (uint32_t)a0 * lbo + (uint32_t)ks * 2048u, lbo, 1024);
+                            umma(tmem_base + buf * 256u, ad, bd, idesc, ks != 0);
+                        }
+                        umma_commit(full_bar(buf));
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ load / move / store warps
+        const int tid = threadIdx.x;           // 0 .. 255
+        const int quarter = warp & 3, group = warp >> 2;
+        const int row = quarter * 32 + lane;    // TMEM lane = row of D this thread reads
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int32_t N = P.n_in, L = P.n_keep, N1 = P.n1, N2 = P.n2, L1 = P.l1, L2 = P.l2, T1 = P.t1, T3 = P.t3;
+        // per-thread constants of the three re-indexing passes
+        const int ri = (row >> 4) & 1;                       // stages 1 and 3: rows 16..31 of a warp are imaginary parts
+        const int32_t cidx = (row >> 5) * 16 + (row & 15);   // t1 (stage 1) or j2 (stage 3) of this row
+        DctmmRow2 meta = {0, 0, 0, 0};
+        if (row < P.rows2) meta = reinterpret_cast<const DctmmRow2*>(static_cast<const uint8_t*>(P.image) + P.f_bytes)[row];
+        const int32_t hL = (L + 1) / 2;
+        const int64_t row_bytes = view.stride_token * 2;
+
+        auto slab_base = [&](int32_t slab) -> char* {
+            const int32_t mat = slab / prm.slabs_per_matrix, piece = slab - mat * prm.slabs_per_matrix;
+            const int32_t tensor = mat / view.mats_per_tensor;
+            return static_cast<char*>(tensor_base(view, tensor)) +
+                   (matrix_offset(view, mat - tensor * view.mats_per_tensor) + (int64_t)prm.sink * view.stride_token) * 2 +
+                   piece * 16;
+        };
+        // Row n of the signal goes to position p of the reordered sequence, p = N2 n1 + n2: piece (k = n1, o = n2).
+        auto issue_loads = [&](int32_t slab) {
+            const char* src = slab_base(slab);
+            const uint32_t dst = base + P.st[0].b_off;
+            const uint32_t k_pad = (uint32_t)P.st[0].k_pad;
+            for (int32_t n = tid; n < N; n += EPI_THREADS) {
+                const int32_t p = (n & 1) ? N - 1 - (n >> 1) : (n >> 1);
+                int32_t n1, n2;
+                divmod_small(p, N2, prm.inv_n2, &n1, &n2);
+                cp_async_16(dst + b_piece((uint32_t)n1, (uint32_t)n2, k_pad), src + (int64_t)n * row_bytes);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        // Rows k .. k_pad-1 of a B buffer are contraction padding: zero for every outer value.
+        auto zero_pad_rows = [&](const DctmmStage& st) {
+            const int32_t pad = st.k_pad - st.k, cols = st.atoms * 8;
+            const uint32_t dst = base + st.b_off;
+            for (int32_t i = tid; i < pad * cols; i += EPI_THREADS) {
+                const int32_t kk = i / cols, o = i - kk * cols;
+                st_shared_16(dst + b_piece((uint32_t)(st.k + kk), (uint32_t)o, (uint32_t)st.k_pad), make_uint4(0u, 0u, 0u, 0u));
+            }
+        };
+
+        uint32_t q = 0;
+        bool alive = true;
+        if (n_iter > 0) issue_loads((int32_t)blockIdx.x);
+        for (int32_t it = 0; it < n_iter && alive; ++it) {
+            const int32_t slab = (int32_t)blockIdx.x + it * (int32_t)gridDim.x;
+            // stage 1 operand: the loads of this slab, issued one slab ahead
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            zero_pad_rows(P.st[0]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(ready_bar(0));
+            char* const out_base = slab_base(slab);
+
+            for (int s = 0; s < 4 && alive; ++s) {
+                const DctmmStage& st = P.st[s];
+                const DctmmStage& nx = P.st[(s + 1) & 3];
+                const uint32_t nb = base + nx.b_off, nk_pad = (uint32_t)nx.k_pad;
+                if (s < 3) zero_pad_rows(nx);
+                for (int32_t a0 = 0; a0 < st.atoms && alive; a0 += CHUNK_ATOMS, ++q) {
+                    const uint32_t buf = q & 1u;
+                    if (!mbar_wait(full_bar(buf), (q >> 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) {
+                        alive = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    // every product of stage 3 has read its operand: that buffer takes the next slab
+                    if (s == 2 && a0 + CHUNK_ATOMS >= st.atoms && it + 1 < n_iter) issue_loads(slab + (int32_t)gridDim.x);
+                    const int32_t n_atoms = min(CHUNK_ATOMS, st.atoms - a0);
+                    for (int32_t a = group; a < n_atoms; a += 2) {
+#pragma unroll 1
+                        for (int half = 0; half < 2; ++half) {
+                            const int32_t o0 = (a0 + a) * 8 + half * 4;  // first outer value of these 32 columns
+                            if (o0 >= st.outer) continue;                 // (warp-uniform)
+                            float v[32];
+                            tmem_ld32(lane_taddr + buf * 256u + (uint32_t)(a * 64 + half * 32), v);
+                            if (s == 0 || s == 2) {
+                                // complex twiddle: this row holds one part, the row 16 lanes away the other
+                                const int32_t den = (s == 0) ? 2 * N : 2 * L;
+                                const int32_t count = (s == 0) ? T1 : L2;
+                                float wr, wi, sr, si;
+                                {
+                                    // phase of column o: stage 1: -pi t1 (4 o + 1) / (2N); stage 3: +pi (4 j2 + 1) o / (2L)
+                                    const int32_t mult = (s == 0) ? (4 * o0 + 1) : o0;
+                                    const int32_t fac = (s == 0) ? cidx : (4 * cidx + 1);
+                                    const int32_t num = (int32_t)(((int64_t)fac * mult) % (2 * den));
+                                    sincos_ratio(num, den, &wi, &wr);
+                                    const int32_t step = (int32_t)(((int64_t)fac * ((s == 0) ? 4 : 1)) % (2 * den));
+                                    sincos_ratio(step, den, &si, &sr);
+                                    if (s == 0) {
+                                        wi = -wi;
+                                        si = -si;
+                                    }
+                                }
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    float out[8];
+                                    const float swi = ri ? wi : -wi;
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c) {
+                                        const float other = __shfl_xor_sync(0xffffffffu, v[j * 8 + c], 16);
+                                        out[c] = fmaf(v[j * 8 + c], wr, other * swi);
+                                    }
+                                    const int32_t o = o0 + j;
+                                    if (cidx < count && o < st.outer) {
+                                        const uint32_t k = (uint32_t)(2 * o + ri);
+                                        st_shared_16(nb + b_piece(k, (uint32_t)cidx, nk_pad), pack8(out));
+                                    }
+                                    const float nr = fmaf(wr, sr, -wi * si), ni = fmaf(wr, si, wi * sr);
+                                    wr = nr;
+                                    wi = ni;
+                                }
+                            } else if (s == 1) {
+                                // retained spectrum values go where stage 3 contracts them
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const int32_t o = o0 + j;
+                                    if (o >= meta.lo && o < meta.hi) {
+                                        const int32_t t = meta.t_start + meta.dir * o;
+                                        const uint4 val = pack8(&v[j * 8]);
+                                        int32_t qa, ra;
+                                        divmod_small(t, L1, prm.inv_l1, &qa, &ra);
+                                        if (ra < T3) st_shared_16(nb + b_piece((uint32_t)qa, (uint32_t)ra, nk_pad), val);
+                                        if (t >= 1) {
+                                            divmod_small(L - t, L1, prm.inv_l1, &qa, &ra);
+                                            if (ra < T3) st_shared_16(nb + b_piece((uint32_t)(L2 + qa), (uint32_t)ra, nk_pad), val);
+                                        } else {
+                                            // h_L = 0: the partner of component 0 in the Hermitian form
+                                            st_shared_16(nb + b_piece((uint32_t)L2, 0u, nk_pad), make_uint4(0u, 0u, 0u, 0u));
+                                        }
+                                    }
+                                }
+                            } else {
+                                // output rows: r_j = y_2j for j < ceil(L/2), r_{L-1-j} = y_{2j+1}
+                                if (row < L1) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        const int32_t o = o0 + j;
+                                        if (o < L2) {
+                                            const int32_t jj = L2 * row + o;
+                                            const int32_t m = jj < hL ? 2 * jj : 2 * (L - 1 - jj) + 1;
+                                            *reinterpret_cast<uint4*>(out_base + (int64_t)m * row_bytes) = pack8(&v[j * 8]);
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar(buf));
+                }
+                if (s < 3 && alive) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(ready_bar(s + 1));
+                }
+            }
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == EPI_WARPS) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS));
+    }
+}
+
+// ---------------------------------------------------------------------------------- host side
+
+inline int32_t round_up(int32_t x, int32_t m) { return (x + m - 1) / m * m; }
+
+uint16_t to_bf16(double x)
+{
+    const float f = (float)x;
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    const uint32_t rounded = u + 0x7fffu + ((u >> 16) & 1u);  // nearest even (inputs are finite)
+    return (uint16_t)(rounded >> 16);
+}
+
+// Stage shapes and shared-memory layout of one factor choice; false when a limit is exceeded.
+bool shape_plan(int32_t N, int32_t L, int32_t n1, int32_t n2, int32_t l1, int32_t l2, DctmmPlan* p, std::vector<DctmmRow2>* rows2)
+{
+    const int32_t t1 = n1 / 2 + 1, t3 = l1 / 2 + 1;
+    if (t1 > 64 || l2 > 64 || l1 > 128) return false;
+    // stage-2 rows: real parts (t = t1 + n1 t2 < L) and negated imaginary parts (t = N - t1 - n1 t2 < L,
+    // only for t1 whose mirror is not computed as a real part: 1 <= t1 < ceil(n1 / 2))
+    rows2->clear();
+    for (int32_t t2 = 0; t2 < n2 && n1 * t2 < L; ++t2) rows2->push_back({n1 * t2, +1, 0, std::min(t1, L - n1 * t2)});
+    const int32_t hi = (n1 + 1) / 2;
+    for (int32_t t2 = 0; t2 < n2; ++t2) {
+        const int32_t lo = std::max(1, N - n1 * t2 - L + 1);
+        if (lo < hi) rows2->push_back({N - n1 * t2, -1, lo, hi});
+    }
+    if ((int32_t)rows2->size() > 128 || rows2->empty()) return false;
+    *p = DctmmPlan();
+    p->n_in = N; p->n_keep = L; p->n1 = n1; p->n2 = n2; p->l1 = l1; p->l2 = l2; p->t1 = t1; p->t3 = t3;
+    p->rows2 = (int32_t)rows2->size();
+    const int32_t k[4] = {n1, 2 * n2, 2 * l2, 2 * t3};
+    const int32_t rows[4] = {32 * ((t1 + 15) / 16), p->rows2, 32 * ((l2 + 15) / 16), l1};
+    const int32_t outer[4] = {n2, t1, t3, l2};
+    int32_t off = 0, b_bytes[4];
+    for (int s = 0; s < 4; ++s) {
+        DctmmStage& st = p->st[s];
+        st.k = k[s];
+        st.k_pad = round_up(k[s], 16);
+        st.rows = rows[s];
+        st.rows8 = round_up(rows[s], 8);
+        st.outer = outer[s];
+        st.atoms = (outer[s] + 7) / 8;
+        st.a_off = off;
+        off += ((st.k_pad + 63) / 64) * st.rows8 * 128;
+        b_bytes[s] = st.atoms * st.k_pad * 128;
+    }
+    p->f_bytes = off;
+    const int32_t x = std::max(b_bytes[0], b_bytes[2]), y = std::max(b_bytes[1], b_bytes[3]);
+    p->st[0].b_off = p->st[2].b_off = off;
+    p->st[1].b_off = p->st[3].b_off = off + x;
+    // an instruction reads 128 rows of a tile of F whatever `rows` is: keep that inside the allocation
+    p->bar_off = std::max(off + x + y, p->st[3].a_off + ((p->st[3].k_pad + 63) / 64 - 1) * p->st[3].rows8 * 128 + 128 * 128);
+    p->bar_off = round_up(p->bar_off, 16);
+    p->smem_bytes = p->bar_off + 128 + 1024;  // barriers, tensor-memory slot, abort flag; alignment slack
+    return p->smem_bytes <= SMEM_LIMIT;
+}
+
+// Rough cycles per slab of a factor choice: 2 k_pad per 64-column group on the tensor pipe, about
+// 20 per outer value in the passes that move the accumulators.
+int64_t plan_cost(const DctmmPlan& p)
+{
+    int64_t c = 0;
+    for (int s = 0; s < 4; ++s) c += 2 * (int64_t)p.st[s].k_pad * p.st[s].atoms + 20 * (int64_t)p.st[s].outer;
+    return c;
+}
+
+}  // namespace
+
+bool dctmm_host_plan(int32_t N, int32_t L, DctmmHostPlan* out)
+{
+    if (N < 16 || N > MAX_N || L < 2 || L >= N) return false;
+    int64_t best = -1;
+    DctmmPlan cand;
+    std::vector<DctmmRow2> rows2;
+    for (int32_t n1 = 1; n1 <= N; ++n1) {
+        if (N % n1) continue;
+        for (int32_t l1 = 1; l1 <= L; ++l1) {
+            if (L % l1) continue;
+            if (!shape_plan(N, L, n1, N / n1, l1, L / l1, &cand, &rows2)) continue;
+            const int64_t c = plan_cost(cand);
+            if (best < 0 || c < best) {
+                best = c;
+                out->plan = cand;
+                out->rows2 = rows2;
+            }
+        }
+    }
+    if (best < 0) return false;
+    const DctmmPlan& p = out->plan;
+    const int32_t n1 = p.n1, n2 = p.n2, l1 = p.l1, l2 = p.l2, t1 = p.t1, t3 = p.t3;
+    const double pi = 3.14159265358979323846;
+    // exact angle reduction: cos / sin of 2 pi a / b with the integer a reduced modulo b first
+    auto cs = [&](int64_t a, int64_t b, double* c, double* s) {
+        a %= b;
+        if (a < 0) a += b;
+        *c = std::cos(2.0 * pi * (double)a / (double)b);
+        *s = std::sin(2.0 * pi * (double)a / (double)b);
+    };
+    for (int s = 0; s < 4; ++s) out->f[s].assign((size_t)p.st[s].rows8 * p.st[s].k_pad, 0.0);
+    // F1: rows (t1, part) in the lane order of the twiddle pass: within every 32 rows, 16 real parts then
+    // the 16 imaginary parts of the same t1.  exp(-2 pi i n1 t1 / N1)
+    for (int32_t r = 0; r < p.st[0].rows; ++r) {
+        const int32_t part = (r >> 4) & 1, t = (r >> 5) * 16 + (r & 15);
+        if (t >= t1) continue;
+        for (int32_t k = 0; k < n1; ++k) {
+            double c, s;
+            cs((int64_t)k * t, n1, &c, &s);
+            out->f[0][(size_t)r * p.st[0].k_pad + k] = part ? -s : c;
+        }
+    }
+    // F2: row (part, t2), columns (n2, re | im) interleaved.  c = (2/N) exp(-i pi t2 / (2 N2)) exp(-2 pi i n2 t2 / N2)
+    // = (2/N) exp(-2 pi i t2 (4 n2 + 1) / (4 N2));  real part of c A: cr Ar - ci Ai;  minus imaginary part: -ci Ar - cr Ai
+    for (int32_t r = 0; r < p.rows2; ++r) {
+        const DctmmRow2& m = out->rows2[r];
+        const int32_t t2 = m.dir > 0 ? m.t_start / n1 : (N - m.t_start) / n1;
+        for (int32_t k = 0; k < n2; ++k) {
+            double c, s;
+            cs((int64_t)t2 * (4 * k + 1), 4 * (int64_t)n2, &c, &s);
+            const double cr = 2.0 / N * c, ci = -2.0 / N * s;
+            double* row = &out->f[1][(size_t)r * p.st[1].k_pad];
+            if (m.dir > 0) {
+                row[2 * k] = cr;
+                row[2 * k + 1] = -ci;
+            } else {
+                row[2 * k] = -ci;
+                row[2 * k + 1] = -cr;
+            }
+        }
+    }
+    // F3: rows (j2, part) in the lane order of the twiddle pass; columns (a | b, t2).
+    // g = exp(i pi t2 / (2 L2)) exp(2 pi i j2 t2 / L2) / 2 = exp(2 pi i t2 (4 j2 + 1) / (4 L2)) / 2;
+    // (a - i b) g: real part a gr + b gi, imaginary part a gi - b gr
+    for (int32_t r = 0; r < p.st[2].rows; ++r) {
+        const int32_t part = (r >> 4) & 1, j2 = (r >> 5) * 16 + (r & 15);
+        if (j2 >= l2) continue;
+        double* row = &out->f[2][(size_t)r * p.st[2].k_pad];
+        for (int32_t k = 0; k < l2; ++k) {
+            double c, s;
+            cs((int64_t)k * (4 * j2 + 1), 4 * (int64_t)l2, &c, &s);
+            const double gr = 0.5 * c, gi = 0.5 * s;
+            row[k] = part ? gi : gr;
+            row[l2 + k] = part ? -gr : gi;
+        }
+    }
+    // F4: row j1, columns (t1, re | im) interleaved: w (cos(2 pi j1 t1 / L1) Cr - sin(2 pi j1 t1 / L1) Ci),
+    // w = 1 for the self-conjugate t1 (0, and L1/2 when L1 is even), 2 otherwise
+    for (int32_t r = 0; r < l1; ++r) {
+        double* row = &out->f[3][(size_t)r * p.st[3].k_pad];
+        for (int32_t k = 0; k < t3; ++k) {
+            double c, s;
+            cs((int64_t)r * k, l1, &c, &s);
+            const double w = (k == 0 || 2 * k == l1) ? 1.0 : 2.0;
+            row[2 * k] = w * c;
+            row[2 * k + 1] = -w * s;
+        }
+    }
+    return true;
+}
+
+void dctmm_host_apply(const DctmmHostPlan& hp, const double* x, int32_t C, double* y)
+{
+    const DctmmPlan& p = hp.plan;
+    const int32_t N = p.n_in, L = p.n_keep, n1 = p.n1, n2 = p.n2, l1 = p.l1, l2 = p.l2, t1 = p.t1, t3 = p.t3;
+    const double pi = 3.14159265358979323846;
+    auto stage = [&](int s, const std::vector<double>& b, std::vector<double>* d) {
+        // d[r][o][c] = sum_k F[r][k] b[k][o][c]
+        const DctmmStage& st = p.st[s];
+        d->assign((size_t)st.rows8 * st.outer * C, 0.0);
+        for (int32_t r = 0; r < st.rows; ++r)
+            for (int32_t k = 0; k < st.k; ++k) {
+                const double f = hp.f[s][(size_t)r * st.k_pad + k];
+                if (f == 0.0) continue;
+                for (int32_t i = 0; i < st.outer * C; ++i) (*d)[(size_t)r * st.outer * C + i] += f * b[(size_t)k * st.outer * C + i];
+            }
+    };
+    std::vector<double> b, d;
+    // load: row n -> reordered position -> (k = n1 index, o = n2 index)
+    b.assign((size_t)n1 * n2 * C, 0.0);
+    for (int32_t n = 0; n < N; ++n) {
+        const int32_t pos = (n & 1) ? N - 1 - (n >> 1) : (n >> 1);
+        const int32_t k = pos / n2, o = pos % n2;
+        for (int32_t c = 0; c < C; ++c) b[((size_t)k * n2 + o) * C + c] = x[(size_t)n * C + c];
+    }
+    stage(0, b, &d);
+    // twiddle pass of stage 1 -> operand of stage 2: k = 2 n2 + part, o = t1
+    b.assign((size_t)2 * n2 * t1 * C, 0.0);
+    for (int32_t r = 0; r < p.st[0].rows; ++r) {
+        const int32_t part = (r >> 4) & 1, t = (r >> 5) * 16 + (r & 15);
+        if (t >= t1) continue;
+        for (int32_t o = 0; o < n2; ++o) {
+            const double ang = -pi * (double)(((int64_t)t * (4 * o + 1)) % (4 * (int64_t)N)) / (2.0 * N);
+            const double wr = std::cos(ang), wi = std::sin(ang);
+            for (int32_t c = 0; c < C; ++c) {
+                const double v = d[((size_t)r * n2 + o) * C + c], other = d[((size_t)(r ^ 16) * n2 + o) * C + c];
+                b[((size_t)(2 * o + part) * t1 + t) * C + c] = v * wr + other * (part ? wi : -wi);
+            }
+        }
+    }
+    stage(1, b, &d);
+    // retained components -> operand of stage 3: k = (a | b) * L2 + t2', o = t1'
+    b.assign((size_t)2 * l2 * t3 * C, 0.0);
+    for (int32_t r = 0; r < p.rows2; ++r) {
+        const DctmmRow2& m = hp.rows2[r];
+        for (int32_t o = m.lo; o < m.hi; ++o) {
+            const int32_t t = m.t_start + m.dir * o;
+            for (int32_t c = 0; c < C; ++c) {
+                const double v = d[((size_t)r * t1 + o) * C + c];
+                if (t % l1 < t3) b[((size_t)(t / l1) * t3 + t % l1) * C + c] = v;
+                if (t >= 1 && (L - t) % l1 < t3) b[((size_t)(l2 + (L - t) / l1) * t3 + (L - t) % l1) * C + c] = v;
+            }
+        }
+    }
+    stage(2, b, &d);
+    // twiddle pass of stage 3 -> operand of stage 4: k = 2 t1' + part, o = j2
+    b.assign((size_t)2 * t3 * l2 * C, 0.0);
+    for (int32_t r = 0; r < p.st[2].rows; ++r) {
+        const int32_t part = (r >> 4) & 1, j2 = (r >> 5) * 16 + (r & 15);
+        if (j2 >= l2) continue;
+        for (int32_t o = 0; o < t3; ++o) {
+            const double ang = pi * (double)(((int64_t)(4 * j2 + 1) * o) % (4 * (int64_t)L)) / (2.0 * L);
+            const double wr = std::cos(ang), wi = std::sin(ang);
+            for (int32_t c = 0; c < C; ++c) {
+                const double v = d[((size_t)r * t3 + o) * C + c], other = d[((size_t)(r ^ 16) * t3 + o) * C + c];
+                b[((size_t)(2 * o + part) * l2 + j2) * C + c] = v * wr + other * (part ? wi : -wi);
+            }
+        }
+    }
+    stage(3, b, &d);
+    const int32_t hL = (L + 1) / 2;
+    for (int32_t r = 0; r < l1; ++r)
+        for (int32_t o = 0; o < l2; ++o) {
+            const int32_t j = l2 * r + o, m = j < hL ? 2 * j : 2 * (L - 1 - j) + 1;
+            for (int32_t c = 0; c < C; ++c) y[(size_t)m * C + c] = d[((size_t)r * l2 + o) * C + c];
+        }
+}
+
+bool dctmm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_keep)
+{
+    if (dtype != FREQKV_BF16 || head_dim % 8 != 0 || n_in < 256) return false;
+    DctmmPlan p;
+    std::vector<DctmmRow2> rows2;
+    if (n_in > MAX_N || n_keep < 2 || n_keep >= n_in) return false;
+    for (int32_t n1 = 1; n1 <= n_in; ++n1) {
+        if (n_in % n1) continue;
+        for (int32_t l1 = 1; l1 <= n_keep; ++l1)
+            if (n_keep % l1 == 0 && shape_plan(n_in, n_keep, n1, n_in / n1, l1, n_keep / l1, &p, &rows2)) return true;
+    }
+    return false;
+}
+
+cudaError_t dctmm_make_plan(int32_t n_in, int32_t n_keep, cudaStream_t stream, DctmmPlan* out)
+{
+    DctmmHostPlan hp;
+    if (!dctmm_host_plan(n_in, n_keep, &hp)) return cudaErrorInvalidValue;
+    DctmmPlan p = hp.plan;
+    const size_t bytes = (size_t)p.f_bytes + hp.rows2.size() * sizeof(DctmmRow2);
+    std::vector<uint8_t> image(bytes, 0);
+    for (int s = 0; s < 4; ++s) {
+        const DctmmStage& st = p.st[s];
+        for (int32_t m = 0; m < st.rows8; ++m)
+            for (int32_t k = 0; k < st.k_pad; ++k) {
+                const uint16_t v = to_bf16(hp.f[s][(size_t)m * st.k_pad + k]);
+                const size_t off = (size_t)st.a_off + (size_t)(k / 64) * st.rows8 * 128 + (size_t)m * 128 +
+                                   ((((k % 64) / 8) ^ (m % 8)) << 4) + (k % 8) * 2;
+                std::memcpy(&image[off], &v, 2);
+            }
+    }
+    std::memcpy(&image[p.f_bytes], hp.rows2.data(), hp.rows2.size() * sizeof(DctmmRow2));
+    void* dev = nullptr;
+    cudaError_t e = cudaMalloc(&dev, bytes);
+    if (e != cudaSuccess) return e;
+    // pageable source: the copy has left the host buffer when the call returns
+    e = cudaMemcpyAsync(dev, image.data(), bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) {
+        cudaFree(dev);
+        return e;
+    }
+    p.image = dev;
+    *out = p;
+    return cudaSuccess;
+}
+
+void dctmm_free_plan(DctmmPlan* plan)
+{
+    if (plan->image) cudaFree(plan->image);
+    plan->image = nullptr;
+}
+
+cudaError_t launch_dctmm(const CacheView& view, int32_t n_mat, const DctmmPlan& plan, int32_t sink, int32_t* status_dev,
+                         unsigned long long wait_limit_ns, int sm_count, cudaStream_t stream)
+{
+    static PerDeviceOnce attrs;
+    const cudaError_t attr_error = attrs.run([] {
+        return cudaFuncSetAttribute(freqkv_dctmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT + 1024);
+    });
+    if (attr_error != cudaSuccess) return attr_error;
+    DctmmParams prm;
+    prm.plan = plan;
+    prm.sink = sink;
+    prm.slabs_per_matrix = view.head_dim / 8;
+    const int64_t total = (int64_t)n_mat * prm.slabs_per_matrix;
+    if (total > 0x7fffffff) return cudaErrorInvalidValue;
+    prm.total_slabs = (int32_t)total;
+    prm.inv_n2 = 1.0f / (float)plan.n2;
+    prm.inv_l1 = 1.0f / (float)plan.l1;
+    prm.status = status_dev;
+    prm.wait_limit_ns = wait_limit_ns;
+    const unsigned grid = (unsigned)std::min<int64_t>(total, sm_count);
+    freqkv_dctmm_kernel<<<grid, THREADS, plan.smem_bytes, stream>>>(view, prm);
+    return cudaGetLastError();
+}
+
+}  // namespace freqkv

@@ -122,7 +122,8 @@ def ar1_rows(
         scaled = x.view(nb, b, w.layers, w.kv_heads, w.head_dim) * scales
         out[:, :, :, n0:n0 + nb, :] = scaled.permute(1, 2, 3, 0, 4).to(w.dtype)
         n0 += nb
-    state = state.view(b, w.layers, w.kv_heads, w.head_dim)
+    if state is not None:
+        state = state.view(b, w.layers, w.kv_heads, w.head_dim)
     return out, state
 
 

@@ -51,7 +51,12 @@ typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
  *         kept_len x n_in projection basis and run on the tcgen05 tensor cores (bf16 caches,
  *         head_dim 128 only); halved by the even/odd symmetry of the cosines after a fold pass
  *         over the cache, or, for kept_len <= 256, straight from the cache without that pass;
- *   FDCT  fast-transform kernel (power-of-two n_in and kept_len only);
+ *   FDCT  fast transform, O(N log N) (Appendix A: the DCT "can be computed using the FFT"): for
+ *         bf16 caches the transform pair is factored into four small dense stages that run on
+ *         the tensor cores, for every n_in = N1 N2 and kept_len = L1 L2 whose factors fit the
+ *         kernel (N1 <= 126, L2 <= 64, L1 <= 128, about 2 kept_len / N1 <= 128, a shared-memory
+ *         budget: n_in up to about 4600 -- 4096 -> 2048 and the paper's 4092 -> 2046 among them),
+ *         in place with no scratch; fp32 caches: a radix-16 kernel for power-of-two lengths;
  *   SIMT  the same projection on the fp32 CUDA cores (any shape; the only path for fp32
  *         caches of non-power-of-two length);
  *   AUTO  picks per shape from a table filled from measurements. */
@@ -315,6 +320,16 @@ freqkv_status freqkv_check_attend(const freqkv_layout* layout, const void* k, co
 freqkv_status freqkv_check_attend_prefill(const freqkv_layout* layout, const void* k, const void* v, int32_t layer,
                                           const void* q, const void* out, int32_t q_heads_per_kv, int32_t n_new,
                                           const int32_t* lens);
+
+/* Host-only diagnostic of the fast transform's plan (no device, no context): applies the
+ * factored chain the FDCT variant would run for (n_in, n_keep) -- same factor choice, same
+ * matrices before rounding, same index maps -- in fp64 on the host to `channels` signals
+ * x[n * channels + c], n < n_in, and writes y[m * channels + c], m < n_keep.  It exists so that a
+ * plan can be checked against the definition (Section 3.3, Eq. 2-3; Appendix A) without a GPU; it
+ * is not a compute path.  factors (optional) receives N1, N2, L1, L2.  UNSUPPORTED when no
+ * factorisation of these lengths fits the kernel. */
+freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, const double* x, int32_t channels, double* y,
+                                          int32_t* factors);
 
 /* Text of the most recent CUDA failure or device-status report seen by this context (owned by
  * the context, valid until its next call); "" if none. */

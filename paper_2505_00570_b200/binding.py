@@ -30,7 +30,7 @@ EXPORTS = [
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
     "freqkv_attend_prefill", "freqkv_check_attend_prefill",
     "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
-    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait",
+    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait", "freqkv_fast_plan_apply_host",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.freqkv_check_attend_prefill.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, I32P]
         L.freqkv_set_wait_limit.argtypes = [c_void_p, c_int64]
         L.freqkv_selftest_bounded_wait.argtypes = [c_void_p, c_int64, c_void_p]
+        L.freqkv_fast_plan_apply_host.argtypes = [c_int32, c_int32, c_void_p, c_int32, c_void_p, I32P]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -162,6 +163,22 @@ def check_attend_prefill(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_p
                          n_new: int, lens) -> int:
     arr = (c_int32 * len(lens))(*lens)
     return lib().freqkv_check_attend_prefill(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, n_new, arr)
+
+
+def fast_plan_apply_host(x, n_keep: int):
+    """``freqkv_fast_plan_apply_host``: the FDCT variant's factored chain applied in fp64 on the
+    host to a float64 numpy array ``x`` [n_in, channels] (a plan diagnostic, not a compute path).
+    Returns (y [n_keep, channels], (N1, N2, L1, L2)); raises FreqKVError(ERR_UNSUPPORTED) when
+    the lengths do not factor within the kernel's limits."""
+    import numpy as np
+
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty((n_keep, x.shape[1]), dtype=np.float64)
+    fac = (c_int32 * 4)()
+    st = lib().freqkv_fast_plan_apply_host(x.shape[0], n_keep, x.ctypes.data, x.shape[1], y.ctypes.data, fac)
+    if st != OK:
+        raise FreqKVError(st, f"freqkv_fast_plan_apply_host: {status_string(st)}")
+    return y, tuple(fac)
 
 
 def _stream_ptr(stream) -> int:

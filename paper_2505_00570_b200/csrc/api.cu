@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "fdct.cuh"
+#include "dctmm.cuh"
 #include "attend.cuh"
 #include "prefill.cuh"
 
@@ -27,6 +28,8 @@ struct freqkv_ctx {
     freqkv_variant forced = FREQKV_AUTO;
     std::map<std::tuple<int32_t, int32_t, int32_t>, Basis> bases;  // (n_in, n_keep, first retained component)
     std::map<std::pair<int32_t, int32_t>, FdctPlan> fdct_plans;
+    std::map<std::pair<int32_t, int32_t>, DctmmPlan> dctmm_plans;
+    std::map<std::pair<int32_t, int32_t>, bool> dctmm_fits;  // does a factorisation of (n_in, n_keep) meet the kernel's limits
     size_t basis_bytes = 0;
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
@@ -198,14 +201,28 @@ bool fdct_applicable(const freqkv_layout& l, int32_t n_in, int32_t n_keep)
     return fdct_supported(l.dtype, l.head_dim, n_in, n_keep) && is_pow2(n_in) && is_pow2(n_keep);
 }
 
+// The fast transform as tensor-core stages: bf16 caches whose lengths factor within the kernel's limits.
+bool dctmm_applicable(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
+{
+    if (l.dtype != FREQKV_BF16 || l.head_dim % 8 != 0) return false;
+    const auto key = std::make_pair(n_in, n_keep);
+    auto it = ctx->dctmm_fits.find(key);
+    if (it != ctx->dctmm_fits.end()) return it->second;
+    const bool ok = dctmm_supported(l.dtype, l.head_dim, n_in, n_keep);
+    if (ctx->dctmm_fits.size() > 4096) ctx->dctmm_fits.clear();
+    ctx->dctmm_fits[key] = ok;
+    return ok;
+}
+
 // Variant table, from measurements on B200 (7B shape, 2048 matrices): at 4096 -> 2048 bf16 the
 // tensor-core projection takes 2.36 ms (fold pass included) and the fast transform 4.63 ms, so
 // bf16 caches with head_dim 128 go to the tensor cores whenever a tile can be filled; the fast
 // transform serves the power-of-two shapes the tensor-core path does not take (fp32 caches, other
 // head sizes); everything else runs as a projection on the CUDA cores.
-int32_t resolve(const freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
+int32_t resolve(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 {
-    const bool g = gemm_applicable(l, n_in, n_keep), f = fdct_applicable(l, n_in, n_keep);
+    const bool g = gemm_applicable(l, n_in, n_keep);
+    const bool f = fdct_applicable(l, n_in, n_keep) || dctmm_applicable(ctx, l, n_in, n_keep);
     switch (ctx->forced) {
         case FREQKV_GEMM: return g ? FREQKV_GEMM : -1;
         case FREQKV_FDCT: return f ? FREQKV_FDCT : -1;
@@ -391,6 +408,26 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
     const CacheView view = make_view(l, k, v, batch0, batch_count);
     const int32_t n_mat = 2 * view.mats_per_tensor;
 
+    if (variant == FREQKV_FDCT && first == 0 && dctmm_applicable(ctx, l, n_in, n_keep)) {
+        DctmmPlan plan;
+        const auto key = std::make_pair(n_in, n_keep);
+        auto it = ctx->dctmm_plans.find(key);
+        if (it == ctx->dctmm_plans.end()) {
+            const cudaError_t e = dctmm_make_plan(n_in, n_keep, stream, &plan);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "dctmm_make_plan");
+            ctx->dctmm_plans[key] = plan;
+        } else {
+            plan = it->second;
+        }
+        cudaError_t e;
+        {
+            TransformTimer timer(ctx, stream);
+            e = launch_dctmm(view, n_mat, plan, sink, ctx->status_dev, ctx->gemm.wait_limit_ns, ctx->sm_count, stream);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "launch_dctmm");
+        ctx->kernels_launched += 1;
+        return FREQKV_OK;
+    }
     if (variant == FREQKV_FDCT) {
         FdctPlan plan;
         const auto key = std::make_pair(n_in, n_keep);
@@ -530,6 +567,7 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx)
     cudaDeviceSynchronize();
     free_bases(ctx);
     for (auto& kv : ctx->fdct_plans) fdct_free_plan(&kv.second);
+    for (auto& kv : ctx->dctmm_plans) dctmm_free_plan(&kv.second);
     gemm_release(&ctx->gemm);
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
@@ -582,6 +620,16 @@ freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (variant == FREQKV_FDCT && dtype == FREQKV_BF16 && n_keep < n_in && dctmm_supported(dtype, 128, n_in, n_keep)) {
+        const auto key = std::make_pair(n_in, n_keep);
+        if (ctx->dctmm_plans.find(key) == ctx->dctmm_plans.end()) {
+            DctmmPlan plan;
+            const cudaError_t e = dctmm_make_plan(n_in, n_keep, stream, &plan);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "dctmm_make_plan");
+            ctx->dctmm_plans[key] = plan;
+        }
+        return FREQKV_OK;
+    }
     if (variant == FREQKV_FDCT) {
         if (!is_pow2(n_in) || !is_pow2(n_keep) || !fdct_supported(dtype, 128, n_in, n_keep)) return FREQKV_ERR_UNSUPPORTED;
         const auto key = std::make_pair(n_in, n_keep);
@@ -1236,6 +1284,22 @@ freqkv_status freqkv_selftest_bounded_wait(freqkv_ctx* ctx, int64_t nanoseconds,
     const cudaError_t e = launch_wait_probe(ctx->status_dev, (unsigned long long)nanoseconds, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bounded wait probe");
     ctx->kernels_launched += 1;
+    return FREQKV_OK;
+}
+
+freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, const double* x, int32_t channels, double* y,
+                                          int32_t* factors)
+{
+    if (!x || !y || channels < 1 || n_in < 1 || n_keep < 1 || n_keep >= n_in) return FREQKV_ERR_INVALID_ARG;
+    DctmmHostPlan hp;
+    if (!dctmm_host_plan(n_in, n_keep, &hp)) return FREQKV_ERR_UNSUPPORTED;
+    if (factors) {
+        factors[0] = hp.plan.n1;
+        factors[1] = hp.plan.n2;
+        factors[2] = hp.plan.l1;
+        factors[3] = hp.plan.l2;
+    }
+    dctmm_host_apply(hp, x, channels, y);
     return FREQKV_OK;
 }
 

@@ -219,8 +219,6 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int32_t* status = prm.status;
-    (void)status;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) mbar_init(ready_bar(s), EPI_THREADS);
@@ -288,6 +286,10 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                     }
                 }
             }
+            if (*abort_flag) {  // products may still be in flight: let them finish before tensor memory is freed
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 1000000ull) __nanosleep(1000);
+            }
         }
     } else {
         // ------------------------------------------------------------ load / move / store warps
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
         const int quarter = warp & 3, group = warp >> 2;
         const int row = quarter * 32 + lane;    // TMEM lane = row of D this thread reads
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int32_t N = P.n_in, L = P.n_keep, N1 = P.n1, N2 = P.n2, L1 = P.l1, L2 = P.l2, T1 = P.t1, T3 = P.t3;
+        const int32_t N = P.n_in, L = P.n_keep, N2 = P.n2, L1 = P.l1, L2 = P.l2, T1 = P.t1, T3 = P.t3;
         // per-thread constants of the three re-indexing passes
         const int ri = (row >> 4) & 1;                       // stages 1 and 3: rows 16..31 of a warp are imaginary parts
         const int32_t cidx = (row >> 5) * 16 + (row & 15);   // t1 (stage 1) or j2 (stage 3) of this row
@@ -528,28 +530,46 @@ int64_t plan_cost(const DctmmPlan& p)
     return c;
 }
 
-}  // namespace
+std::vector<int32_t> divisors(int32_t n)
+{
+    std::vector<int32_t> d;
+    for (int32_t i = 1; (int64_t)i * i <= n; ++i)
+        if (n % i == 0) {
+            d.push_back(i);
+            if (i != n / i) d.push_back(n / i);
+        }
+    std::sort(d.begin(), d.end());
+    return d;
+}
 
-bool dctmm_host_plan(int32_t N, int32_t L, DctmmHostPlan* out)
+// The cheapest factor choice that meets every limit; false if there is none.
+bool choose_factors(int32_t N, int32_t L, DctmmPlan* plan, std::vector<DctmmRow2>* rows2_out)
 {
     if (N < 16 || N > MAX_N || L < 2 || L >= N) return false;
     int64_t best = -1;
     DctmmPlan cand;
     std::vector<DctmmRow2> rows2;
-    for (int32_t n1 = 1; n1 <= N; ++n1) {
-        if (N % n1) continue;
-        for (int32_t l1 = 1; l1 <= L; ++l1) {
-            if (L % l1) continue;
+    const std::vector<int32_t> dn = divisors(N), dl = divisors(L);
+    for (int32_t n1 : dn) {
+        if (n1 / 2 + 1 > 64) continue;
+        for (int32_t l1 : dl) {
             if (!shape_plan(N, L, n1, N / n1, l1, L / l1, &cand, &rows2)) continue;
             const int64_t c = plan_cost(cand);
             if (best < 0 || c < best) {
                 best = c;
-                out->plan = cand;
-                out->rows2 = rows2;
+                *plan = cand;
+                *rows2_out = rows2;
             }
         }
     }
-    if (best < 0) return false;
+    return best >= 0;
+}
+
+}  // namespace
+
+bool dctmm_host_plan(int32_t N, int32_t L, DctmmHostPlan* out)
+{
+    if (!choose_factors(N, L, &out->plan, &out->rows2)) return false;
     const DctmmPlan& p = out->plan;
     const int32_t n1 = p.n1, n2 = p.n2, l1 = p.l1, l2 = p.l2, t1 = p.t1, t3 = p.t3;
     const double pi = 3.14159265358979323846;
@@ -703,13 +723,7 @@ bool dctmm_supported(int32_t dtype, int32_t head_dim, int32_t n_in, int32_t n_ke
     if (dtype != FREQKV_BF16 || head_dim % 8 != 0 || n_in < 256) return false;
     DctmmPlan p;
     std::vector<DctmmRow2> rows2;
-    if (n_in > MAX_N || n_keep < 2 || n_keep >= n_in) return false;
-    for (int32_t n1 = 1; n1 <= n_in; ++n1) {
-        if (n_in % n1) continue;
-        for (int32_t l1 = 1; l1 <= n_keep; ++l1)
-            if (n_keep % l1 == 0 && shape_plan(n_in, n_keep, n1, n_in / n1, l1, n_keep / l1, &p, &rows2)) return true;
-    }
-    return false;
+    return choose_factors(n_in, n_keep, &p, &rows2);
 }
 
 cudaError_t dctmm_make_plan(int32_t n_in, int32_t n_keep, cudaStream_t stream, DctmmPlan* out)

@@ -48,18 +48,18 @@
 namespace freqkv {
 namespace {
 
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 16;                // four per TMEM lane quarter: one atom of a chunk each
 constexpr int EPI_THREADS = EPI_WARPS * 32;
 constexpr int THREADS = EPI_THREADS + 32;
 constexpr int CHUNK_ATOMS = 4;                 // 4 x 64 columns = N 256 per instruction
 constexpr int TMEM_COLS = 512;
 constexpr int SMEM_LIMIT = 232448 - 1024;      // opt-in maximum minus alignment slack
-constexpr int MAX_N = 8192;
+constexpr int MAX_LOADS = 9;                 // rows per loading thread
+constexpr int MAX_N = MAX_LOADS * EPI_THREADS;
 
 struct DctmmParams {
     DctmmPlan plan;
     int32_t sink, slabs_per_matrix, total_slabs;
-    float inv_n2, inv_l1;
     int32_t* status;
     unsigned long long wait_limit_ns;
 };
@@ -93,22 +93,40 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// The same, but the thread may be suspended for up to `hint_ns` while the phase is incomplete
+// (it is woken when the phase completes): a waiting warp then leaves the issue slots to the others.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
 // Wait for the phase with the given parity; gives up when another thread has raised the abort
 // flag or after limit_ns (then it sets the status bit and raises the flag).  False = gave up.
+// The global timer is read rarely: its reads are slow and many warps wait at once.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
                                           unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > limit_ns) {
-            atomicOr(status, DCTMM_ERR_WAIT);
-            *abort_flag = 1;
-            __threadfence_block();
-            return false;
+    unsigned long long t0 = 0;
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
+        if ((spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > limit_ns) {
+                atomicOr(status, DCTMM_ERR_WAIT);
+                *abort_flag = 1;
+                __threadfence_block();
+                return false;
+            }
         }
     }
 }
@@ -186,15 +204,6 @@ __host__ __device__ __forceinline__ uint32_t b_piece(uint32_t k, uint32_t o, uin
     return (o >> 3) * (k_pad * 128u) + k * 128u + (((o & 7u) ^ (k & 7u)) << 4);
 }
 
-// q = t / d, r = t % d for 0 <= t < 2^15, 1 <= d <= 2^8 through one multiplication (exact: the
-// half added to t keeps the product at least 0.5 / d away from an integer, far more than the
-// rounding of a float product of this size).
-__device__ __forceinline__ void divmod_small(int32_t t, int32_t d, float inv_d, int32_t* q, int32_t* r)
-{
-    *q = (int32_t)(((float)t + 0.5f) * inv_d);
-    *r = t - *q * d;
-}
-
 // cos and sin of pi * num / den for integers 0 <= num < 2 den.
 __device__ __forceinline__ void sincos_ratio(int32_t num, int32_t den, float* s, float* c)
 {
@@ -233,14 +242,16 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
-    // the matrices F: a plain copy of the pre-swizzled image; both data buffers start as zeros
-    // (never-written padding must not hold NaN bit patterns: it meets zero entries of F)
+    // the matrices F and the destination table of the second pass: plain copies of the host-built
+    // image; both data buffers start as zeros (never-written padding must not hold NaN bit
+    // patterns: it meets zero entries of F)
     {
         const uint4* img = static_cast<const uint4*>(P.image);
         uint4* dst = reinterpret_cast<uint4*>(aligned);
-        const int32_t n_f = P.f_bytes / 16, n_all = P.bar_off / 16;
+        const int32_t n_f = P.f_bytes / 16, n_data = P.tab_off / 16, n_tab = P.tab_bytes / 16;
         for (int32_t i = threadIdx.x; i < n_f; i += THREADS) dst[i] = img[i];
-        for (int32_t i = n_f + threadIdx.x; i < n_all; i += THREADS) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (int32_t i = n_f + threadIdx.x; i < n_data; i += THREADS) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (int32_t i = threadIdx.x; i < n_tab; i += THREADS) dst[n_data + i] = img[n_f + i];
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -293,18 +304,50 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
         }
     } else {
         // ------------------------------------------------------------ load / move / store warps
-        const int tid = threadIdx.x;           // 0 .. 255
-        const int quarter = warp & 3, group = warp >> 2;
+        const int tid = threadIdx.x;            // 0 .. EPI_THREADS - 1
+        const int quarter = warp & 3, group = warp >> 2;  // group g takes atom g of every 4-atom chunk
         const int row = quarter * 32 + lane;    // TMEM lane = row of D this thread reads
         const uint32_t lane_taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int32_t N = P.n_in, L = P.n_keep, N2 = P.n2, L1 = P.l1, L2 = P.l2, T1 = P.t1, T3 = P.t3;
-        // per-thread constants of the three re-indexing passes
+        const int32_t N = P.n_in, L = P.n_keep, N2 = P.n2, L2 = P.l2, T1 = P.t1;
         const int ri = (row >> 4) & 1;                       // stages 1 and 3: rows 16..31 of a warp are imaginary parts
         const int32_t cidx = (row >> 5) * 16 + (row & 15);   // t1 (stage 1) or j2 (stage 3) of this row
-        DctmmRow2 meta = {0, 0, 0, 0};
-        if (row < P.rows2) meta = reinterpret_cast<const DctmmRow2*>(static_cast<const uint8_t*>(P.image) + P.f_bytes)[row];
         const int32_t hL = (L + 1) / 2;
         const int64_t row_bytes = view.stride_token * 2;
+
+        // Rows this thread loads (n = tid + EPI_THREADS * i) and where each 16-byte piece goes:
+        // row n is position p of the reordered sequence, p = N2 n1 + n2: piece (k = n1, o = n2).
+        uint32_t load_dst[MAX_LOADS];
+#pragma unroll
+        for (int i = 0; i < MAX_LOADS; ++i) {
+            const int32_t n = tid + EPI_THREADS * i;
+            const int32_t p = (n & 1) ? N - 1 - (n >> 1) : (n >> 1);
+            load_dst[i] = n < N ? base + P.st[0].b_off + b_piece((uint32_t)(p / N2), (uint32_t)(p % N2), (uint32_t)P.st[0].k_pad) : 0u;
+        }
+        // Twiddles of the two complex passes, by recurrence: this thread's value at the first outer
+        // index of its first atom (o = 8 * group), the factor from o to o + 1, and the factor over
+        // the 24 outer values of the other groups' atoms in between.
+        // stage 1: exp(-i pi t1 (4 o + 1) / (2N));  stage 3: exp(+i pi (4 j2 + 1) o / (2L)).
+        float2 tw_start[2], tw_step1[2], tw_jump[2];
+        uint32_t swz[4];  // stages 1, 3 write row k = 2 o + ri, piece cidx % 8 of its atom: the swizzled piece for o % 4 = j
+#pragma unroll
+        for (int j = 0; j < 4; ++j) swz[j] = ((((uint32_t)cidx & 7u) ^ ((uint32_t)(2 * j + ri) & 7u)) << 4) + (uint32_t)ri * 128u;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int32_t den = i == 0 ? 2 * N : 2 * L;         // angles are pi * num / den, num taken modulo 2 den
+            const int32_t fac = i == 0 ? cidx : 4 * cidx + 1;   // the row's own factor of the phase
+            const int32_t per_o = i == 0 ? 4 : 1;               // phase units per step of o
+            const int32_t first = i == 0 ? 4 * (8 * group) + 1 : 8 * group;
+            auto unit = [&](int32_t mult) {
+                float sn, cs;
+                sincos_ratio((int32_t)(((int64_t)fac * mult) % (2 * den)), den, &sn, &cs);
+                return make_float2(cs, i == 0 ? -sn : sn);
+            };
+            tw_start[i] = unit(first);
+            tw_step1[i] = unit(per_o);
+            tw_jump[i] = unit(24 * per_o);
+        }
+        const bool row2_ok = row < P.rows2;  // rows of stage 2 that exist: the table has no others
+        const uint32_t* dest_tab = reinterpret_cast<const uint32_t*>(aligned + P.tab_off) + (row2_ok ? row : 0) * (P.st[1].atoms * 8);
 
         auto slab_base = [&](int32_t slab) -> char* {
             const int32_t mat = slab / prm.slabs_per_matrix, piece = slab - mat * prm.slabs_per_matrix;
@@ -313,46 +356,46 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                    (matrix_offset(view, mat - tensor * view.mats_per_tensor) + (int64_t)prm.sink * view.stride_token) * 2 +
                    piece * 16;
         };
-        // Row n of the signal goes to position p of the reordered sequence, p = N2 n1 + n2: piece (k = n1, o = n2).
-        auto issue_loads = [&](int32_t slab) {
-            const char* src = slab_base(slab);
-            const uint32_t dst = base + P.st[0].b_off;
-            const uint32_t k_pad = (uint32_t)P.st[0].k_pad;
-            for (int32_t n = tid; n < N; n += EPI_THREADS) {
-                const int32_t p = (n & 1) ? N - 1 - (n >> 1) : (n >> 1);
-                int32_t n1, n2;
-                divmod_small(p, N2, prm.inv_n2, &n1, &n2);
-                cp_async_16(dst + b_piece((uint32_t)n1, (uint32_t)n2, k_pad), src + (int64_t)n * row_bytes);
+        auto issue_loads = [&](const char* src) {
+            const char* p = src + (int64_t)tid * row_bytes;
+#pragma unroll
+            for (int i = 0; i < MAX_LOADS; ++i) {
+                if (tid + EPI_THREADS * i < N) cp_async_16(load_dst[i], p);
+                p += (int64_t)EPI_THREADS * row_bytes;
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
-        // Rows k .. k_pad-1 of a B buffer are contraction padding: zero for every outer value.
+        // Rows k .. k_pad-1 of a B buffer are contraction padding: zero for every outer value
+        // (thread: outer value tid % 64, rows tid / 64, + 8, ...; at most 64 outer values per buffer...)
         auto zero_pad_rows = [&](const DctmmStage& st) {
-            const int32_t pad = st.k_pad - st.k, cols = st.atoms * 8;
+            const int32_t cols = st.atoms * 8;
             const uint32_t dst = base + st.b_off;
-            for (int32_t i = tid; i < pad * cols; i += EPI_THREADS) {
-                const int32_t kk = i / cols, o = i - kk * cols;
-                st_shared_16(dst + b_piece((uint32_t)(st.k + kk), (uint32_t)o, (uint32_t)st.k_pad), make_uint4(0u, 0u, 0u, 0u));
-            }
+            for (int32_t o = tid & 63; o < cols; o += 64)
+                for (int32_t k = st.k + (tid >> 6); k < st.k_pad; k += EPI_THREADS / 64)
+                    st_shared_16(dst + b_piece((uint32_t)k, (uint32_t)o, (uint32_t)st.k_pad), make_uint4(0u, 0u, 0u, 0u));
         };
 
         uint32_t q = 0;
         bool alive = true;
-        if (n_iter > 0) issue_loads((int32_t)blockIdx.x);
+        char* cur_base = n_iter > 0 ? slab_base((int32_t)blockIdx.x) : nullptr;
+        char* next_base = cur_base;
+        if (n_iter > 0) issue_loads(cur_base);
         for (int32_t it = 0; it < n_iter && alive; ++it) {
             const int32_t slab = (int32_t)blockIdx.x + it * (int32_t)gridDim.x;
+            cur_base = next_base;
             // stage 1 operand: the loads of this slab, issued one slab ahead
             asm volatile("cp.async.wait_all;" ::: "memory");
             zero_pad_rows(P.st[0]);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(ready_bar(0));
-            char* const out_base = slab_base(slab);
 
             for (int s = 0; s < 4 && alive; ++s) {
                 const DctmmStage& st = P.st[s];
                 const DctmmStage& nx = P.st[(s + 1) & 3];
                 const uint32_t nb = base + nx.b_off, nk_pad = (uint32_t)nx.k_pad;
                 if (s < 3) zero_pad_rows(nx);
+                const bool quarter_active = quarter * 32 < st.rows;  // rows past the stage's own are never read
+                float wr = tw_start[s >> 1].x, wi = tw_start[s >> 1].y;
                 for (int32_t a0 = 0; a0 < st.atoms && alive; a0 += CHUNK_ATOMS, ++q) {
                     const uint32_t buf = q & 1u;
                     if (!mbar_wait(full_bar(buf), (q >> 1) & 1, abort_flag, prm.status, prm.wait_limit_ns)) {
@@ -361,33 +404,23 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                     }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     // every product of stage 3 has read its operand: that buffer takes the next slab
-                    if (s == 2 && a0 + CHUNK_ATOMS >= st.atoms && it + 1 < n_iter) issue_loads(slab + (int32_t)gridDim.x);
-                    const int32_t n_atoms = min(CHUNK_ATOMS, st.atoms - a0);
-                    for (int32_t a = group; a < n_atoms; a += 2) {
-#pragma unroll 1
-                        for (int half = 0; half < 2; ++half) {
-                            const int32_t o0 = (a0 + a) * 8 + half * 4;  // first outer value of these 32 columns
-                            if (o0 >= st.outer) continue;                 // (warp-uniform)
-                            float v[32];
-                            tmem_ld32(lane_taddr + buf * 256u + (uint32_t)(a * 64 + half * 32), v);
-                            if (s == 0 || s == 2) {
-                                // complex twiddle: this row holds one part, the row 16 lanes away the other
-                                const int32_t den = (s == 0) ? 2 * N : 2 * L;
-                                const int32_t count = (s == 0) ? T1 : L2;
-                                float wr, wi, sr, si;
-                                {
-                                    // phase of column o: stage 1: -pi t1 (4 o + 1) / (2N); stage 3: +pi (4 j2 + 1) o / (2L)
-                                    const int32_t mult = (s == 0) ? (4 * o0 + 1) : o0;
-                                    const int32_t fac = (s == 0) ? cidx : (4 * cidx + 1);
-                                    const int32_t num = (int32_t)(((int64_t)fac * mult) % (2 * den));
-                                    sincos_ratio(num, den, &wi, &wr);
-                                    const int32_t step = (int32_t)(((int64_t)fac * ((s == 0) ? 4 : 1)) % (2 * den));
-                                    sincos_ratio(step, den, &si, &sr);
-                                    if (s == 0) {
-                                        wi = -wi;
-                                        si = -si;
-                                    }
-                                }
+                    if (s == 2 && a0 + CHUNK_ATOMS >= st.atoms && it + 1 < n_iter) {
+                        next_base = slab_base(slab + (int32_t)gridDim.x);
+                        issue_loads(next_base);
+                    }
+                    if (quarter_active && a0 + group < st.atoms) {
+                        const uint32_t taddr = lane_taddr + buf * 256u + (uint32_t)(group * 64);
+                        const int32_t o_atom = (a0 + group) * 8;  // first outer value of this thread's atom
+                        if (s == 0 || s == 2) {
+                            // complex twiddle: this row holds one part, the row 16 lanes away the other
+                            const int32_t count = (s == 0) ? T1 : L2;
+                            const float sr = tw_step1[s >> 1].x, si = tw_step1[s >> 1].y;
+                            const bool mine = cidx < count;
+                            const uint32_t dst0 = nb + ((uint32_t)cidx >> 3) * (nk_pad * 128u) + (uint32_t)o_atom * 256u;
+#pragma unroll
+                            for (int half = 0; half < 2; ++half) {
+                                float v[32];
+                                tmem_ld32(taddr + half * 32, v);
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
                                     float out[8];
@@ -397,45 +430,56 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                                         const float other = __shfl_xor_sync(0xffffffffu, v[j * 8 + c], 16);
                                         out[c] = fmaf(v[j * 8 + c], wr, other * swi);
                                     }
-                                    const int32_t o = o0 + j;
-                                    if (cidx < count && o < st.outer) {
-                                        const uint32_t k = (uint32_t)(2 * o + ri);
-                                        st_shared_16(nb + b_piece(k, (uint32_t)cidx, nk_pad), pack8(out));
-                                    }
+                                    if (mine && o_atom + half * 4 + j < st.outer)
+                                        st_shared_16(dst0 + (uint32_t)(half * 4 + j) * 256u + swz[j], pack8(out));
                                     const float nr = fmaf(wr, sr, -wi * si), ni = fmaf(wr, si, wi * sr);
                                     wr = nr;
                                     wi = ni;
                                 }
-                            } else if (s == 1) {
-                                // retained spectrum values go where stage 3 contracts them
+                            }
+                            {   // now at o_atom + 8: skip the other groups' atoms, on to o_atom + 32
+                                const float jr = tw_jump[s >> 1].x, ji = tw_jump[s >> 1].y;
+                                const float nr = fmaf(wr, jr, -wi * ji), ni = fmaf(wr, ji, wi * jr);
+                                wr = nr;
+                                wi = ni;
+                            }
+                        } else if (s == 1) {
+                            // retained spectrum values go where stage 3 contracts them: up to two places
+                            // each, from the host-built table (16-bit piece numbers, 0xffff = nowhere)
+#pragma unroll
+                            for (int half = 0; half < 2; ++half) {
+                                if (o_atom + half * 4 >= st.outer) continue;
+                                float v[32];
+                                tmem_ld32(taddr + half * 32, v);
+                                const uint4 dd = *reinterpret_cast<const uint4*>(dest_tab + o_atom + half * 4);
+                                const uint32_t d[4] = {dd.x, dd.y, dd.z, dd.w};
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
-                                    const int32_t o = o0 + j;
-                                    if (o >= meta.lo && o < meta.hi) {
-                                        const int32_t t = meta.t_start + meta.dir * o;
+                                    const uint32_t da = d[j] & 0xffffu, db = d[j] >> 16;
+                                    if (row2_ok && d[j] != 0xffffffffu) {
                                         const uint4 val = pack8(&v[j * 8]);
-                                        int32_t qa, ra;
-                                        divmod_small(t, L1, prm.inv_l1, &qa, &ra);
-                                        if (ra < T3) st_shared_16(nb + b_piece((uint32_t)qa, (uint32_t)ra, nk_pad), val);
-                                        if (t >= 1) {
-                                            divmod_small(L - t, L1, prm.inv_l1, &qa, &ra);
-                                            if (ra < T3) st_shared_16(nb + b_piece((uint32_t)(L2 + qa), (uint32_t)ra, nk_pad), val);
-                                        } else {
-                                            // h_L = 0: the partner of component 0 in the Hermitian form
-                                            st_shared_16(nb + b_piece((uint32_t)L2, 0u, nk_pad), make_uint4(0u, 0u, 0u, 0u));
-                                        }
+                                        if (da != 0xffffu) st_shared_16(nb + da * 16u, val);
+                                        if (db != 0xffffu) st_shared_16(nb + db * 16u, val);
                                     }
                                 }
-                            } else {
-                                // output rows: r_j = y_2j for j < ceil(L/2), r_{L-1-j} = y_{2j+1}
-                                if (row < L1) {
+                            }
+                            // h_L = 0: the partner of component 0 in the Hermitian form
+                            if (row == 0 && o_atom == 0) st_shared_16(nb + b_piece((uint32_t)L2, 0u, nk_pad), make_uint4(0u, 0u, 0u, 0u));
+                        } else {
+                            // output rows: r_j = y_2j for j < ceil(L/2), r_{L-1-j} = y_{2j+1}
+#pragma unroll
+                            for (int half = 0; half < 2; ++half) {
+                                if (o_atom + half * 4 >= st.outer) continue;
+                                float v[32];
+                                tmem_ld32(taddr + half * 32, v);
+                                if (row < P.l1) {
 #pragma unroll
                                     for (int j = 0; j < 4; ++j) {
-                                        const int32_t o = o0 + j;
+                                        const int32_t o = o_atom + half * 4 + j;
                                         if (o < L2) {
                                             const int32_t jj = L2 * row + o;
                                             const int32_t m = jj < hL ? 2 * jj : 2 * (L - 1 - jj) + 1;
-                                            *reinterpret_cast<uint4*>(out_base + (int64_t)m * row_bytes) = pack8(&v[j * 8]);
+                                            *reinterpret_cast<uint4*>(cur_base + (int64_t)m * row_bytes) = pack8(&v[j * 8]);
                                         }
                                     }
                                 }
@@ -516,7 +560,10 @@ bool shape_plan(int32_t N, int32_t L, int32_t n1, int32_t n2, int32_t l1, int32_
     p->st[1].b_off = p->st[3].b_off = off + x;
     // an instruction reads 128 rows of a tile of F whatever `rows` is: keep that inside the allocation
     p->bar_off = std::max(off + x + y, p->st[3].a_off + ((p->st[3].k_pad + 63) / 64 - 1) * p->st[3].rows8 * 128 + 128 * 128);
-    p->bar_off = round_up(p->bar_off, 16);
+    // destination table of the second pass: one 32-bit entry per (row, outer value of stage 2)
+    p->tab_off = round_up(p->bar_off, 16);
+    p->tab_bytes = round_up(p->rows2 * p->st[1].atoms * 8 * 4, 16);
+    p->bar_off = p->tab_off + p->tab_bytes;
     p->smem_bytes = p->bar_off + 128 + 1024;  // barriers, tensor-memory slot, abort flag; alignment slack
     return p->smem_bytes <= SMEM_LIMIT;
 }
@@ -731,7 +778,7 @@ cudaError_t dctmm_make_plan(int32_t n_in, int32_t n_keep, cudaStream_t stream, D
     DctmmHostPlan hp;
     if (!dctmm_host_plan(n_in, n_keep, &hp)) return cudaErrorInvalidValue;
     DctmmPlan p = hp.plan;
-    const size_t bytes = (size_t)p.f_bytes + hp.rows2.size() * sizeof(DctmmRow2);
+    const size_t bytes = (size_t)p.f_bytes + p.tab_bytes;
     std::vector<uint8_t> image(bytes, 0);
     for (int s = 0; s < 4; ++s) {
         const DctmmStage& st = p.st[s];
@@ -743,7 +790,24 @@ cudaError_t dctmm_make_plan(int32_t n_in, int32_t n_keep, cudaStream_t stream, D
                 std::memcpy(&image[off], &v, 2);
             }
     }
-    std::memcpy(&image[p.f_bytes], hp.rows2.data(), hp.rows2.size() * sizeof(DctmmRow2));
+    // where the value of row r, column o of stage 2 goes in the operand of stage 3 (16-byte piece
+    // numbers): as a_{t2'} of column t mod L1 and / or as b_{t2'} of column (L - t) mod L1
+    {
+        const int32_t cols = p.st[1].atoms * 8, k3_pad = p.st[2].k_pad;
+        std::vector<uint32_t> tab((size_t)p.tab_bytes / 4, 0xffffffffu);
+        for (int32_t r = 0; r < p.rows2; ++r) {
+            const DctmmRow2& m = hp.rows2[r];
+            for (int32_t o = m.lo; o < m.hi; ++o) {
+                const int32_t t = m.t_start + m.dir * o;
+                uint32_t da = 0xffffu, db = 0xffffu;
+                if (t % p.l1 < p.t3) da = b_piece((uint32_t)(t / p.l1), (uint32_t)(t % p.l1), (uint32_t)k3_pad) / 16;
+                if (t >= 1 && (p.n_keep - t) % p.l1 < p.t3)
+                    db = b_piece((uint32_t)(p.l2 + (p.n_keep - t) / p.l1), (uint32_t)((p.n_keep - t) % p.l1), (uint32_t)k3_pad) / 16;
+                tab[(size_t)r * cols + o] = da | (db << 16);
+            }
+        }
+        std::memcpy(&image[p.f_bytes], tab.data(), (size_t)p.tab_bytes);
+    }
     void* dev = nullptr;
     cudaError_t e = cudaMalloc(&dev, bytes);
     if (e != cudaSuccess) return e;
@@ -779,8 +843,6 @@ cudaError_t launch_dctmm(const CacheView& view, int32_t n_mat, const DctmmPlan& 
     const int64_t total = (int64_t)n_mat * prm.slabs_per_matrix;
     if (total > 0x7fffffff) return cudaErrorInvalidValue;
     prm.total_slabs = (int32_t)total;
-    prm.inv_n2 = 1.0f / (float)plan.n2;
-    prm.inv_l1 = 1.0f / (float)plan.l1;
     prm.status = status_dev;
     prm.wait_limit_ns = wait_limit_ns;
     const unsigned grid = (unsigned)std::min<int64_t>(total, sm_count);

@@ -35,8 +35,9 @@ struct DctmmPlan {
     int32_t rows2 = 0;
     int32_t f_bytes = 0;     // bytes of the four F images (start of shared memory)
     int32_t smem_bytes = 0;  // everything: F, two data buffers, barriers
+    int32_t tab_off = 0, tab_bytes = 0;  // destination table of the pass after stage 2 (shared memory)
     int32_t bar_off = 0;
-    void* image = nullptr;   // device: F images (f_bytes) followed by rows2 DctmmRow2 entries
+    void* image = nullptr;   // device: F images (f_bytes) followed by that table
 };
 
 // Largest transform the kernel's shared memory can hold is found by trying: true when some

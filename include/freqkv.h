@@ -147,7 +147,12 @@ freqkv_status freqkv_power_spectrum(freqkv_ctx* ctx, const freqkv_layout* layout
  * each sequence with the transform of its own length (same definition as above with
  * N = lens[b] - sink, L = kept_len[b]).  `lens` and `kept_len` are host arrays of
  * layout->batch entries; on success lens[b] is updated to sink + kept_len[b].  All arguments
- * are validated for every sequence before anything is enqueued. */
+ * are validated for every sequence before anything is enqueued.  When every sequence that needs
+ * work takes the folded tensor-core form (bf16, head_dim 128, more than 256 kept rows) the whole
+ * batch is ONE fold launch and ONE tensor-core launch over a host-built work list (longest
+ * sequences first), all plans built and all memory allocated before the first of them; the folded
+ * inputs of the whole batch then live in the context's scratch (as many bytes as the non-sink
+ * rows; beyond 64 GiB, or with other variants in the batch, the call goes run by run). */
 freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layout, void* k, void* v, int32_t* lens,
                                      const int32_t* kept_len, int32_t sink, void* cuda_stream);
 

@@ -773,6 +773,57 @@ freqkv_status freqkv_compress_ragged(freqkv_ctx* ctx, const freqkv_layout* layou
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     WorkOrder order(ctx, stream);
+    // When every sequence that needs work takes the folded tensor-core form, the whole batch runs
+    // as one fold launch and one tensor-core launch; every plan is built and all memory is
+    // allocated before the first of them.
+    {
+        bool all_folded = true;
+        int32_t active = 0;
+        for (int32_t b = 0; b < layout->batch; ++b) {
+            if (variant[b] == 0) continue;
+            ++active;
+            if (variant[b] != FREQKV_GEMM || gemm_is_direct(kept_len[b])) all_folded = false;
+        }
+        if (all_folded && active > 1) {
+            std::vector<RaggedItem> items;
+            bool ok = true;
+            for (int pass = 0; pass < 2 && ok; ++pass) {  // second pass: a flush of the plan cache may have dropped earlier plans
+                items.clear();
+                for (int32_t b = 0; b < layout->batch && ok; ++b) {
+                    if (variant[b] == 0) continue;
+                    Basis basis;
+                    st = get_basis(ctx, lens[b] - sink, kept_len[b], 0, false, true, stream, &basis);
+                    if (st != FREQKV_OK) return st;  // nothing enqueued but plan builders
+                    items.push_back({b, basis});
+                }
+                bool intact = true;
+                for (const RaggedItem& it : items) {
+                    auto found = ctx->bases.find(std::make_tuple(it.basis.n_in, it.basis.n_keep, (int32_t)0));
+                    if (found == ctx->bases.end() || found->second.fold != it.basis.fold) intact = false;
+                }
+                if (intact) break;
+                if (pass == 1) ok = false;
+            }
+            if (ok) {
+                const CacheView view = make_view(*layout, k, v, 0, layout->batch);
+                TransformTimer timer(ctx, stream, false);
+                LaunchHooks hooks;
+                hooks.user = &timer;
+                hooks.before = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->begin(); };
+                hooks.after = [](void* u, cudaStream_t) { static_cast<TransformTimer*>(u)->end(); };
+                ctx->gemm.last_error = nullptr;
+                const cudaError_t e = launch_gemm_ragged(&ctx->gemm, view, items, sink, ctx->status_dev, ctx->sm_count, hooks, stream);
+                if (e == cudaSuccess) {
+                    ctx->kernels_launched += ctx->gemm.kernels_last_call;
+                    for (int32_t b = 0; b < layout->batch; ++b) lens[b] = sink + kept_len[b];
+                    return FREQKV_OK;
+                }
+                if (e != cudaErrorMemoryAllocation || ctx->gemm.kernels_last_call != 0)
+                    return cuda_fail(ctx, e, ctx->gemm.last_error ? ctx->gemm.last_error : "launch_gemm_ragged");
+                cudaGetLastError();  // the folded batch does not fit: go sequence by sequence
+            }
+        }
+    }
     // Sequences are grouped by runs of equal (length, kept length); each run is one group.
     for (int32_t b = 0; b < layout->batch;) {
         int32_t e = b + 1;

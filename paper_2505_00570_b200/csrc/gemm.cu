@@ -43,6 +43,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <vector>
 
 #include "gemm.cuh"
 
@@ -63,6 +64,10 @@ constexpr unsigned long long LANDING_NS = 1000000ull;        // 1 ms: far longer
 
 constexpr uint32_t ERR_FULL_WAIT = 1u, ERR_EMPTY_WAIT = 2u, ERR_ACC_FULL_WAIT = 4u, ERR_ACC_EMPTY_WAIT = 8u;
 
+struct RaggedSeq {
+    int32_t tile0, pair0, n_keep, rows_half, basis_rows_pad, k_steps, m_pairs, pad;
+};
+
 struct GemmParams {
     int32_t n_keep;             // L
     int32_t rows_half;          // ceil(L / 2): folded output rows
@@ -77,6 +82,21 @@ struct GemmParams {
     int32_t n_in;
     int32_t* status;
     unsigned long long wait_limit_ns;  // bound of every mbarrier wait
+    // ragged mode only: per-sequence shapes (sorted by decreasing work, tile0 = running sum of tiles,
+    // one entry past the end holds the total) and two tensor maps per sequence (basis, folded inputs)
+    const RaggedSeq* seqs;
+    const CUtensorMap* seq_maps;
+    int32_t n_seqs;
+};
+
+// What one tile (256 folded output rows x K|V of one (batch, layer, kv_head)) works on.
+struct TileCtx {
+    const CUtensorMap* map_p;   // basis
+    const CUtensorMap* map_x;   // folded inputs
+    int32_t pair;               // (batch, layer, kv_head) triple inside the cache view
+    int32_t pair_local;         // ... inside the scratch planes its tensor map covers
+    int32_t m_tile;             // which 256 folded rows
+    int32_t n_keep, rows_half, basis_rows_pad, k_steps;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -329,7 +349,49 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
     }
 }
 
+// The same for a ragged batch in one launch: every sequence has the same number of matrices, so
+// block x belongs to job x / mats_per_seq.
+__global__ void __launch_bounds__(256) fold_ragged_kernel(const CacheView view, const FoldJob* jobs, int32_t mats_per_seq)
+{
+    const FoldJob job = jobs[blockIdx.x / mats_per_seq];
+    const uint32_t pt = blockIdx.x % mats_per_seq;
+    const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
+                    (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
+    const int64_t row_bytes = view.stride_token * 2;
+    const uint32_t total = (uint32_t)job.n_half * 16u;
+    uint4* u_plane = job.dst + (int64_t)pt * 2 * total;
+    for (uint32_t c0 = blockIdx.y * 1024u; c0 < total; c0 += gridDim.y * 1024u) {
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4), nr = job.n_in - 1 - n;
+                a[j] = __ldcs(reinterpret_cast<const uint4*>(x + n * row_bytes) + (i & 15u));
+                b[j] = __ldcs(reinterpret_cast<const uint4*>(x + nr * row_bytes) + (i & 15u));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4);
+                uint4 u, v;
+                fold8(a[j], b[j], &u, &v);
+                if (job.n_in - 1 - n == n) {
+                    u = a[j];
+                    v = make_uint4(0u, 0u, 0u, 0u);
+                }
+                __stcs(u_plane + i, u);
+                __stcs(u_plane + total + i, v);
+            }
+        }
+    }
+}
+
 // MODE_FOLD: the compression above.
+// MODE_RAGGED: MODE_FOLD over sequences of different lengths in one launch: a tile looks up its
+//   sequence (shapes, basis and folded-input tensor maps) in a table built on the host.
 // MODE_SPECTRUM: the basis holds the even and the odd rows of the plain N-point DCT-II instead of
 //   Pe and Po, so S and D are the components z_2m and z_2m+1 themselves; the epilogue squares them,
 //   sums over the 128 channels of its tensor and adds the sum to the power spectrum of its
@@ -339,7 +401,42 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
 //   cache (map_x = K tensor, map_v = V tensor, 5-D maps over the non-sink rows), there is one
 //   accumulator and one tile per (batch, layer, kv_head).  The tile's rows are stored only after
 //   every slice of its matrices has been read, so writing in place is safe here too.
-constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2;
+constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2, MODE_RAGGED = 3;
+
+template <int MODE>
+__device__ __forceinline__ TileCtx tile_ctx(const GemmParams& prm, int32_t tile, const CUtensorMap* map_p, const CUtensorMap* map_x)
+{
+    TileCtx t;
+    if constexpr (MODE == MODE_RAGGED) {
+        int32_t lo = 0, hi = prm.n_seqs;  // last sequence whose first tile is <= tile
+        while (hi - lo > 1) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (__ldg(&prm.seqs[mid].tile0) <= tile) lo = mid; else hi = mid;
+        }
+        const RaggedSeq s = prm.seqs[lo];
+        const int32_t local = tile - s.tile0;
+        t.map_p = prm.seq_maps + 2 * lo;
+        t.map_x = prm.seq_maps + 2 * lo + 1;
+        t.pair_local = local / s.m_pairs;
+        t.m_tile = local % s.m_pairs;
+        t.pair = s.pair0 + t.pair_local;
+        t.n_keep = s.n_keep;
+        t.rows_half = s.rows_half;
+        t.basis_rows_pad = s.basis_rows_pad;
+        t.k_steps = s.k_steps;
+    } else {
+        t.map_p = map_p;
+        t.map_x = map_x;
+        t.pair_local = tile / prm.m_pairs;
+        t.m_tile = tile % prm.m_pairs;
+        t.pair = prm.pair0 + t.pair_local;
+        t.n_keep = prm.n_keep;
+        t.rows_half = prm.rows_half;
+        t.basis_rows_pad = prm.basis_rows_pad;
+        t.k_steps = prm.k_steps;
+    }
+    return t;
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -366,7 +463,8 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const uint32_t rank = cluster_rank();  // 0 = leader of the pair
     const int32_t cluster = blockIdx.x / 2, n_clusters = gridDim.x / 2;
-    const int32_t total_tiles = prm.pair_count * prm.m_pairs;  // tiles of 256 folded rows x 256 columns
+    // tiles of 256 folded rows x 256 columns
+    const int32_t total_tiles = MODE == MODE_RAGGED ? prm.seqs[prm.n_seqs].tile0 : prm.pair_count * prm.m_pairs;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -397,14 +495,15 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             uint32_t it = 0;  // global slice counter: stage = it % STAGES, phase = it / STAGES
             bool alive = true;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters) {
-                const int32_t pair_local = tile / prm.m_pairs;
-                const int32_t m0 = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM;
-                const int32_t pair = prm.pair0 + pair_local;  // direct mode: coordinates inside the cache tensor
+                const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x);
+                const int32_t pair_local = tc.pair_local;
+                const int32_t m0 = (tc.m_tile * 2 + (int32_t)rank) * BM;
+                const int32_t pair = tc.pair;  // direct mode: coordinates inside the cache tensor
                 const int32_t head = pair % view.kv_heads, layer = (pair / view.kv_heads) % view.layers,
                               seq = pair / (view.kv_heads * view.layers);
                 for (int eo = 0; eo < PHASES && alive; ++eo) {
                     const int32_t plane = (pair_local * 2 + (int32_t)rank) * 2 + eo;  // rank 0: K channels, rank 1: V
-                    for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
+                    for (int32_t ks = 0; ks < tc.k_steps; ++ks, ++it) {
                         const int s = it % STAGES;
                         if (it >= STAGES &&
                             !mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag, prm.status, ERR_EMPTY_WAIT, prm.wait_limit_ns)) {
@@ -415,14 +514,14 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         const uint32_t leader_full = cluster_addr(full_bar(s), 0);
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
                         const int32_t k0 = ks * BK;
-                        tma_load_2d(stage, &map_p, leader_full, k0, eo * prm.basis_rows_pad + m0);
+                        tma_load_2d(stage, tc.map_p, leader_full, k0, eo * tc.basis_rows_pad + m0);
                         if constexpr (MODE == MODE_DIRECT) {
                             const CUtensorMap* cache = rank ? &map_v : &map_x;
                             tma_load_5d(stage + A_BYTES, cache, leader_full, 0, k0, head, layer, seq);
                             tma_load_5d(stage + A_BYTES + B_CHUNK_BYTES, cache, leader_full, 64, k0, head, layer, seq);
                         } else {
-                            tma_load_3d(stage + A_BYTES, &map_x, leader_full, 0, k0, plane);
-                            tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, &map_x, leader_full, 64, k0, plane);
+                            tma_load_3d(stage + A_BYTES, tc.map_x, leader_full, 0, k0, plane);
+                            tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, tc.map_x, leader_full, 64, k0, plane);
                         }
                     }
                 }
@@ -438,6 +537,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             uint32_t it = 0, tile_no = 0;
             bool alive = true;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters, ++tile_no) {
+                const int32_t k_steps = tile_ctx<MODE>(prm, tile, &map_p, &map_x).k_steps;
                 for (int eo = 0; eo < PHASES && alive; ++eo) {
                     if (tile_no > 0) {  // both CTAs' epilogues must have read this accumulator of the last tile
                         if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT, prm.wait_limit_ns)) {
@@ -446,7 +546,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     }
-                    for (int32_t ks = 0; ks < prm.k_steps; ++ks, ++it) {
+                    for (int32_t ks = 0; ks < k_steps; ++ks, ++it) {
                         const int s = it % STAGES;
                         if (!mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, prm.status, ERR_FULL_WAIT, prm.wait_limit_ns)) {
                             alive = false;
@@ -548,13 +648,13 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             // D = Po V: combine and store rows m and L-1-m
             if (!mbar_wait(acc_full_bar(1), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int32_t pair_local = tile / prm.m_pairs;
-            const int32_t m = ((tile % prm.m_pairs) * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
-            const int32_t mr = prm.n_keep - 1 - m;
-            const bool row_ok = m < prm.rows_half;
+            const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x);
+            const int32_t m = (tc.m_tile * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
+            const int32_t mr = tc.n_keep - 1 - m;
+            const bool row_ok = m < tc.rows_half;
             const float sgn = (float)prm.mirror_sign;
             __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
-                                 matrix_offset(view, prm.pair0 + pair_local) + (int64_t)prm.sink * view.stride_token;
+                                 matrix_offset(view, tc.pair) + (int64_t)prm.sink * view.stride_token;
             uint4* out_p = reinterpret_cast<uint4*>(mat + (int64_t)m * view.stride_token);
             uint4* out_m = reinterpret_cast<uint4*>(mat + (int64_t)mr * view.stride_token);
 #pragma unroll
@@ -655,6 +755,7 @@ bool encode_scratch_map(CUtensorMap* map, void* scratch, int32_t n_half, int32_t
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr size_t kRaggedScratchLimit = size_t(64) << 30;  // a ragged batch is folded whole: beyond this it goes sequence by sequence
 constexpr size_t kFoldBufferBytes = size_t(2304) << 20;  // scratch for the folded inputs: a 7B-shaped cache of 4096 tokens fits in one pass
 
 }  // namespace
@@ -681,6 +782,8 @@ cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, in
             e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_SPECTRUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) {
             state->last_error = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -781,6 +884,9 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         prm.n_in = basis.n_in;
         prm.status = status_dev;
         prm.wait_limit_ns = state->wait_limit_ns;
+        prm.seqs = nullptr;
+        prm.seq_maps = nullptr;
+        prm.n_seqs = 0;
         const int32_t tiles = job.pair_count * m_pairs;
         const int clusters = std::min<int32_t>(tiles, state->max_clusters);
         cudaLaunchConfig_t cfg = {};
@@ -805,6 +911,146 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         }
         state->kernels_last_call += 2;
     }
+    return cudaSuccess;
+}
+
+// A ragged batch in two launches: one fold pass and one tensor-core pass over every sequence,
+// longest first.  Everything that can fail for lack of memory happens before the first launch.
+cudaError_t launch_gemm_ragged(GemmState* state, const CacheView& view, const std::vector<RaggedItem>& items_in, int32_t sink,
+                               int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream)
+{
+    state->kernels_last_call = 0;
+    if (items_in.empty()) return cudaSuccess;
+    const cudaError_t prepared = gemm_prepare(state, 0, items_in[0].basis, sm_count);
+    if (prepared != cudaSuccess) return prepared;
+    const int32_t lh = view.layers * view.kv_heads;  // (layer, kv_head) pairs per sequence
+    std::vector<RaggedItem> items = items_in;
+    auto work = [](const RaggedItem& it) { return (int64_t)it.basis.n_in * it.basis.n_keep; };
+    std::stable_sort(items.begin(), items.end(), [&](const RaggedItem& a, const RaggedItem& b) { return work(a) > work(b); });
+    const size_t n = items.size();
+    // scratch: the folded planes of every sequence, back to back
+    std::vector<size_t> offset(n);
+    size_t total = 0;
+    int32_t max_half = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const int32_t n_half = (items[i].basis.n_in + 1) / 2;
+        offset[i] = total;
+        total += (size_t)lh * 4 * n_half * 256;
+        max_half = std::max(max_half, n_half);
+    }
+    if (total > kRaggedScratchLimit) {
+        state->last_error = "folded inputs of the ragged batch exceed the scratch limit";
+        return cudaErrorMemoryAllocation;
+    }
+    if (total > state->scratch_bytes) {
+        if (state->scratch) {
+            const cudaError_t e = cudaDeviceSynchronize();
+            if (e != cudaSuccess) return e;
+            cudaFree(state->scratch);
+            state->scratch = nullptr;
+            state->scratch_bytes = 0;
+        }
+        const cudaError_t e = cudaMalloc(&state->scratch, total);
+        if (e != cudaSuccess) {
+            state->last_error = "cudaMalloc(fold scratch of a ragged batch)";
+            return e;
+        }
+        state->scratch_bytes = total;
+    }
+    // tables: two tensor maps, one shape record and one fold job per sequence
+    const size_t maps_bytes = n * 2 * sizeof(CUtensorMap), seqs_bytes = (n + 1) * sizeof(RaggedSeq), jobs_bytes = n * sizeof(FoldJob);
+    const size_t meta_bytes = maps_bytes + seqs_bytes + jobs_bytes;
+    if (meta_bytes > state->ragged_meta_bytes) {
+        if (state->ragged_meta) {
+            const cudaError_t e = cudaDeviceSynchronize();
+            if (e != cudaSuccess) return e;
+            cudaFree(state->ragged_meta);
+            state->ragged_meta = nullptr;
+            state->ragged_meta_bytes = 0;
+        }
+        const cudaError_t e = cudaMalloc(&state->ragged_meta, meta_bytes);
+        if (e != cudaSuccess) {
+            state->last_error = "cudaMalloc(tables of a ragged batch)";
+            return e;
+        }
+        state->ragged_meta_bytes = meta_bytes;
+    }
+    std::vector<CUtensorMap> maps(2 * n);
+    std::vector<RaggedSeq> seqs(n + 1);
+    std::vector<FoldJob> jobs(n);
+    int64_t tiles = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const Basis& b = items[i].basis;
+        const int32_t n_half = (b.n_in + 1) / 2, rows_half = (b.n_keep + 1) / 2;
+        char* planes = static_cast<char*>(state->scratch) + offset[i];
+        if (!encode_basis_map(&maps[2 * i], b) || !encode_scratch_map(&maps[2 * i + 1], planes, n_half, lh * 4)) {
+            state->last_error = "tensor map encoding rejected a sequence of the ragged batch";
+            return cudaErrorInvalidValue;
+        }
+        RaggedSeq& s = seqs[i];
+        s.tile0 = (int32_t)tiles;
+        s.pair0 = items[i].batch_index * lh;
+        s.n_keep = b.n_keep;
+        s.rows_half = rows_half;
+        s.basis_rows_pad = b.fold_rows_pad;
+        s.k_steps = (n_half + BK - 1) / BK;
+        s.m_pairs = (rows_half + 2 * BM - 1) / (2 * BM);
+        s.pad = 0;
+        tiles += (int64_t)lh * s.m_pairs;
+        FoldJob& j = jobs[i];
+        j.pair0 = s.pair0;
+        j.pair_count = lh;
+        j.n_in = b.n_in;
+        j.n_half = n_half;
+        j.sink = sink;
+        j.dst = reinterpret_cast<uint4*>(planes);
+    }
+    if (tiles > 0x7fffffff || (int64_t)n * 2 * lh > 0x7fffffff) return cudaErrorInvalidValue;
+    seqs[n] = RaggedSeq{(int32_t)tiles, 0, 0, 0, 0, 0, 1, 0};
+    char* meta = static_cast<char*>(state->ragged_meta);
+    // pageable sources: each copy has left its host buffer when the call returns
+    cudaError_t e = cudaMemcpyAsync(meta, maps.data(), maps_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(meta + maps_bytes, seqs.data(), seqs_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(meta + maps_bytes + seqs_bytes, jobs.data(), jobs_bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return e;
+
+    const unsigned fold_y = (unsigned)std::min<int64_t>(((int64_t)max_half * 16 + 1023) / 1024, 64);
+    fold_ragged_kernel<<<dim3((unsigned)(n * 2 * lh), fold_y), 256, 0, stream>>>(
+        view, reinterpret_cast<const FoldJob*>(meta + maps_bytes + seqs_bytes), 2 * lh);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        state->last_error = "fold_ragged_kernel launch";
+        return e;
+    }
+    GemmParams prm = {};
+    prm.sink = sink;
+    prm.mirror_sign = 1;
+    prm.status = status_dev;
+    prm.wait_limit_ns = state->wait_limit_ns;
+    prm.seq_maps = reinterpret_cast<const CUtensorMap*>(meta);
+    prm.seqs = reinterpret_cast<const RaggedSeq*>(meta + maps_bytes);
+    prm.n_seqs = (int32_t)n;
+    const int clusters = (int)std::min<int64_t>(tiles, state->max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (hooks.before) hooks.before(hooks.user, stream);
+    e = cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_RAGGED>, maps[0], maps[1], maps[1], view, prm);
+    if (hooks.after) hooks.after(hooks.user, stream);
+    if (e != cudaSuccess) {
+        state->last_error = "freqkv_gemm_kernel launch";
+        return e;
+    }
+    state->kernels_last_call = 2;
     return cudaSuccess;
 }
 
@@ -900,6 +1146,9 @@ cudaError_t launch_wait_probe(int32_t* status_dev, unsigned long long limit_ns, 
 
 void gemm_release(GemmState* state)
 {
+    if (state->ragged_meta) cudaFree(state->ragged_meta);
+    state->ragged_meta = nullptr;
+    state->ragged_meta_bytes = 0;
     if (state->scratch) cudaFree(state->scratch);
     state->scratch = nullptr;
     state->scratch_bytes = 0;

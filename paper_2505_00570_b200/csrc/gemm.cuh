@@ -1,5 +1,7 @@
 // Tensor-core (tcgen05) execution of the compression Y = P X: declarations.
 #pragma once
+#include <vector>
+
 #include "common.cuh"
 
 namespace freqkv {
@@ -11,6 +13,8 @@ struct GemmState {
     int max_clusters = 0;     // CTA pairs that can be resident at once
     void* scratch = nullptr;  // folded inputs U, V: [pairs][K|V][U|V][ceil(n_in/2)][128] bf16 per pass
     size_t scratch_bytes = 0;
+    void* ragged_meta = nullptr;  // tensor maps, shapes and fold jobs of a ragged batch (device)
+    size_t ragged_meta_bytes = 0;
     unsigned long long wait_limit_ns = 2000000000ull;  // bound of every mbarrier wait inside the kernel (2 s)
 };
 
@@ -37,6 +41,16 @@ cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, in
 // At most 256 kept rows: one tile per (batch, layer, kv_head), no fold pass, the dense basis (Basis::dense).
 bool gemm_is_direct(int32_t n_keep);
 cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
+                               int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
+// One sequence of a ragged batch: its index in the cache and the (folded) basis of its lengths.
+struct RaggedItem {
+    int32_t batch_index;
+    Basis basis;
+};
+// Every listed sequence in one fold launch and one tensor-core launch (each needs more than 256 kept
+// rows: the folded form).  `view` covers the whole cache.  cudaErrorMemoryAllocation before anything is
+// enqueued when the folded inputs do not fit: the caller then goes sequence by sequence.
+cudaError_t launch_gemm_ragged(GemmState* state, const CacheView& view, const std::vector<RaggedItem>& items, int32_t sink,
                                int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 void gemm_release(GemmState* state);
 // A one-thread kernel that waits, with the tensor-core kernel's own bounded wait, on an mbarrier

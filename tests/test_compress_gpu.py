@@ -189,6 +189,43 @@ def test_ragged_batch_small(ctx):
                 assert torch.equal(t_out[b, 0, h, 4 + kept[b]:], t_in[b, 0, h, 4 + kept[b]:])
 
 
+def test_ragged_batch_in_two_launches(ctx):
+    """A ragged batch whose sequences all take the folded tensor-core form runs as ONE fold launch
+    and ONE tensor-core launch (the kernel counter says so); odd and even lengths, one sequence
+    left alone (kept == length), one with more than one tile of rows.  Against the oracle, against
+    the bytes outside the rewritten rows, and bit for bit against compressing each sequence on
+    its own (same kernels, same arithmetic)."""
+    w = small(cap=1400, dtype=torch.bfloat16, sink=4, B=6, Ly=2, H=3, outliers=2)
+    k, v = synth.make_cache(w, "cuda")
+    k_in, v_in = k.clone(), v.clone()
+    lens = [1400, 523, 1101, 523, 700, 1337]
+    kept = [(n - 4) // 2 for n in lens]
+    kept[4] = 700 - 4          # identity: nothing to do for this sequence
+    ctx.set_variant(fk.AUTO)
+    before = ctx.get_timing()[2]
+    new_lens = ctx.compress_ragged(k, v, lens, kept, 4)
+    assert ctx.last_device_status() == fk.OK
+    launched = ctx.get_timing()[2] - before
+    assert new_lens == [4 + x for x in kept]
+    plans = len({(n, kp) for n, kp in zip(lens, kept) if kp != n - 4})
+    assert launched <= 2 + plans, f"{launched} kernels for the batch (2 + at most {plans} plan builders expected)"
+    before = ctx.get_timing()[2]
+    k2, v2 = k_in.clone(), v_in.clone()
+    assert ctx.compress_ragged(k2, v2, lens, kept, 4) == new_lens
+    assert ctx.get_timing()[2] - before == 2          # plans cached: exactly the two launches
+    assert torch.equal(k2, k) and torch.equal(v2, v)
+    for b in range(6):
+        one_k, one_v = k_in[b:b + 1].clone(), v_in[b:b + 1].clone()
+        ctx.compress(one_k, one_v, lens[b], kept[b], 4)
+        assert torch.equal(one_k[0], k[b]) and torch.equal(one_v[0], v[b]), f"sequence {b} differs from its own compression"
+        for t_in, t_out in ((k_in, k), (v_in, v)):
+            assert torch.equal(t_out[b, :, :, :4], t_in[b, :, :, :4])
+            assert torch.equal(t_out[b, :, :, 4 + kept[b]:], t_in[b, :, :, 4 + kept[b]:])
+            for (l, h) in ((0, 0), (1, 2)):
+                want = oracle.compress_matrix(parity.to_f64(t_in[b, l, h, 4:lens[b]]), kept[b])
+                parity.check_matrix(parity.to_f64(t_out[b, l, h, 4:4 + kept[b]]), want, torch.bfloat16, f"sequence {b}")
+
+
 # ---- tensor-core projection (tcgen05 / TMEM / TMA), bf16 caches with head_dim 128
 @pytest.mark.parametrize("n_in,kept,sink", [(128, 64, 0), (256, 128, 4), (300, 150, 4), (700, 350, 4), (1000, 999, 1),
                                             (1023, 511, 0), (1500, 100, 4), (64, 32, 2), (17, 5, 0)])

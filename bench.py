@@ -234,7 +234,7 @@ def run_ragged(args, ctx, fk, synth, w, dev, peaks):
     for _ in range(args.warmup):
         ctx.compress_ragged(k, v, lens, kept, sink)
     torch.cuda.synchronize()
-    ctx.get_timing()
+    _, _, launched0 = ctx.get_timing()
     ctx.set_timing(True)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
@@ -242,7 +242,7 @@ def run_ragged(args, ctx, fk, synth, w, dev, peaks):
         ctx.compress_ragged(k, v, lens, kept, sink)
     b.record()
     torch.cuda.synchronize()
-    n_launch, t_ms, _ = ctx.get_timing()
+    n_launch, t_ms, launched1 = ctx.get_timing()
     ctx.set_timing(False)
     ms = a.elapsed_time(b) / args.steps
     gemm_ms = t_ms / args.steps
@@ -257,8 +257,10 @@ def run_ragged(args, ctx, fk, synth, w, dev, peaks):
             "roofline": {"bound": "tensor", "achieved": flops / (gemm_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
                          "unit": "TFLOP/s", "frac": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                          "peak_kind": "sustained, of " + peaks["source"], "kernel": "gemm", "kernel_ms": gemm_ms / (n_launch / args.steps),
+                         "frac_of_burst_peak": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                          "launches_per_call": n_launch / args.steps, "traffic": None},
-            "cpu_baseline": None, "e2e": None, "gpu_launches": None}
+            "kernels_per_call": (launched1 - launched0) / args.steps,
+            "cpu_baseline": None, "e2e": None, "gpu_launches": launched1 - launched0}
 
 
 def run_stream_graph(args, ctx, fk, synth, w, dev, peaks, total_tokens=32768):

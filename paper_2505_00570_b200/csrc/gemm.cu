@@ -403,17 +403,26 @@ __global__ void __launch_bounds__(256) fold_ragged_kernel(const CacheView view, 
 //   every slice of its matrices has been read, so writing in place is safe here too.
 constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2, MODE_RAGGED = 3;
 
+// Ragged mode: a role walks its tiles in increasing order, so the sequence a tile belongs to is
+// found by moving a cursor forward; the table is read only when a tile crosses into a new sequence.
+struct SeqCursor {
+    int32_t idx = -1, end_tile = 0;
+    RaggedSeq s;
+};
+
 template <int MODE>
-__device__ __forceinline__ TileCtx tile_ctx(const GemmParams& prm, int32_t tile, const CUtensorMap* map_p, const CUtensorMap* map_x)
+__device__ __forceinline__ TileCtx tile_ctx(const GemmParams& prm, int32_t tile, const CUtensorMap* map_p, const CUtensorMap* map_x,
+                                            SeqCursor& cur)
 {
     TileCtx t;
     if constexpr (MODE == MODE_RAGGED) {
-        int32_t lo = 0, hi = prm.n_seqs;  // last sequence whose first tile is <= tile
-        while (hi - lo > 1) {
-            const int32_t mid = (lo + hi) >> 1;
-            if (__ldg(&prm.seqs[mid].tile0) <= tile) lo = mid; else hi = mid;
+        while (tile >= cur.end_tile) {
+            ++cur.idx;
+            cur.s = prm.seqs[cur.idx];
+            cur.end_tile = __ldg(&prm.seqs[cur.idx + 1].tile0);
         }
-        const RaggedSeq s = prm.seqs[lo];
+        const RaggedSeq& s = cur.s;
+        const int32_t lo = cur.idx;
         const int32_t local = tile - s.tile0;
         t.map_p = prm.seq_maps + 2 * lo;
         t.map_x = prm.seq_maps + 2 * lo + 1;
@@ -494,8 +503,9 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         if (lane == 0) {
             uint32_t it = 0;  // global slice counter: stage = it % STAGES, phase = it / STAGES
             bool alive = true;
+            SeqCursor cursor;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters) {
-                const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x);
+                const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor);
                 const int32_t pair_local = tc.pair_local;
                 const int32_t m0 = (tc.m_tile * 2 + (int32_t)rank) * BM;
                 const int32_t pair = tc.pair;  // direct mode: coordinates inside the cache tensor
@@ -536,8 +546,9 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, tile_no = 0;
             bool alive = true;
+            SeqCursor cursor;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters, ++tile_no) {
-                const int32_t k_steps = tile_ctx<MODE>(prm, tile, &map_p, &map_x).k_steps;
+                const int32_t k_steps = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor).k_steps;
                 for (int eo = 0; eo < PHASES && alive; ++eo) {
                     if (tile_no > 0) {  // both CTAs' epilogues must have read this accumulator of the last tile
                         if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT, prm.wait_limit_ns)) {
@@ -574,6 +585,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + tensor * 128;
         const uint32_t leader_s_empty = cluster_addr(acc_empty_bar(0), 0), leader_d_empty = cluster_addr(acc_empty_bar(1), 0);
         uint32_t tile_no = 0;
+        SeqCursor cursor;
         if constexpr (MODE == MODE_DIRECT) {
             for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
                 if (!mbar_wait(acc_full_bar(0), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) break;
@@ -648,7 +660,7 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             // D = Po V: combine and store rows m and L-1-m
             if (!mbar_wait(acc_full_bar(1), tile_no & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x);
+            const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor);
             const int32_t m = (tc.m_tile * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
             const int32_t mr = tc.n_keep - 1 - m;
             const bool row_ok = m < tc.rows_half;

@@ -568,8 +568,9 @@ bool shape_plan(int32_t N, int32_t L, int32_t n1, int32_t n2, int32_t l1, int32_
     return p->smem_bytes <= SMEM_LIMIT;
 }
 
-// Rough cycles per slab of a factor choice: 2 k_pad per 64-column group on the tensor pipe, about
-// 20 per outer value in the passes that move the accumulators.
+// Rough cycles per slab of a factor choice: 2 k_pad per 64-column atom on the tensor pipe, about
+// 20 per outer value in the passes that move the accumulators.  (Measured on B200, the choices
+// that fit shared memory for 4092 -> 2046 and 4096 -> 2048 all land within 4 % of each other.)
 int64_t plan_cost(const DctmmPlan& p)
 {
     int64_t c = 0;

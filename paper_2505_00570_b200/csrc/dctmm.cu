@@ -160,23 +160,25 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 lanes x 32 consecutive columns of tensor memory into registers.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32])
+// 32 lanes x 16 consecutive columns, issued without waiting; the registers may be read only after
+// tmem_ld_wait16 on the same array (which names them as operands, so that no use is scheduled before it).
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&u)[16])
 {
-    uint32_t u[32];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
-          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
-          "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
-          "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&u)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]), "+r"(u[8]),
+                   "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15])
+                 :
+                 : "memory");
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
@@ -186,6 +188,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __device__ __forceinline__ uint4 pack8(const float* v)
 {
     return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+__device__ __forceinline__ uint4 pack8u(const uint32_t* u)
+{
+    return make_uint4(pack_bf16(__uint_as_float(u[0]), __uint_as_float(u[1])), pack_bf16(__uint_as_float(u[2]), __uint_as_float(u[3])),
+                      pack_bf16(__uint_as_float(u[4]), __uint_as_float(u[5])), pack_bf16(__uint_as_float(u[6]), __uint_as_float(u[7])));
 }
 __device__ __forceinline__ void st_shared_16(uint32_t addr, const uint4& v)
 {
@@ -411,6 +418,10 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                     if (quarter_active && a0 + group < st.atoms) {
                         const uint32_t taddr = lane_taddr + buf * 256u + (uint32_t)(group * 64);
                         const int32_t o_atom = (a0 + group) * 8;  // first outer value of this thread's atom
+                        // The atom's 64 columns come out of tensor memory 16 at a time (two outer values);
+                        // the load of the next 16 is in flight while these are worked on.
+                        uint32_t ua[16], ub[16];
+                        tmem_ld16_issue(taddr, ua);
                         if (s == 0 || s == 2) {
                             // complex twiddle: this row holds one part, the row 16 lanes away the other
                             const int32_t count = (s == 0) ? T1 : L2;
@@ -418,20 +429,23 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                             const bool mine = cidx < count;
                             const uint32_t dst0 = nb + ((uint32_t)cidx >> 3) * (nk_pad * 128u) + (uint32_t)o_atom * 256u;
 #pragma unroll
-                            for (int half = 0; half < 2; ++half) {
-                                float v[32];
-                                tmem_ld32(taddr + half * 32, v);
+                            for (int part = 0; part < 4; ++part) {
+                                uint32_t(&u)[16] = (part & 1) ? ub : ua;
+                                tmem_ld_wait16(u);
+                                if (part < 3) tmem_ld16_issue(taddr + (part + 1) * 16, (part & 1) ? ua : ub);
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
+                                for (int jj = 0; jj < 2; ++jj) {
+                                    const int j = (part & 1) * 2 + jj;  // o % 4
                                     float out[8];
                                     const float swi = ri ? wi : -wi;
 #pragma unroll
                                     for (int c = 0; c < 8; ++c) {
-                                        const float other = __shfl_xor_sync(0xffffffffu, v[j * 8 + c], 16);
-                                        out[c] = fmaf(v[j * 8 + c], wr, other * swi);
+                                        const float val = __uint_as_float(u[jj * 8 + c]);
+                                        const float other = __shfl_xor_sync(0xffffffffu, val, 16);
+                                        out[c] = fmaf(val, wr, other * swi);
                                     }
-                                    if (mine && o_atom + half * 4 + j < st.outer)
-                                        st_shared_16(dst0 + (uint32_t)(half * 4 + j) * 256u + swz[j], pack8(out));
+                                    if (mine && o_atom + part * 2 + jj < st.outer)
+                                        st_shared_16(dst0 + (uint32_t)(part * 2 + jj) * 256u + swz[j], pack8(out));
                                     const float nr = fmaf(wr, sr, -wi * si), ni = fmaf(wr, si, wi * sr);
                                     wr = nr;
                                     wi = ni;
@@ -447,17 +461,17 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                             // retained spectrum values go where stage 3 contracts them: up to two places
                             // each, from the host-built table (16-bit piece numbers, 0xffff = nowhere)
 #pragma unroll
-                            for (int half = 0; half < 2; ++half) {
-                                if (o_atom + half * 4 >= st.outer) continue;
-                                float v[32];
-                                tmem_ld32(taddr + half * 32, v);
-                                const uint4 dd = *reinterpret_cast<const uint4*>(dest_tab + o_atom + half * 4);
-                                const uint32_t d[4] = {dd.x, dd.y, dd.z, dd.w};
+                            for (int part = 0; part < 4; ++part) {
+                                uint32_t(&u)[16] = (part & 1) ? ub : ua;
+                                tmem_ld_wait16(u);
+                                if (part < 3) tmem_ld16_issue(taddr + (part + 1) * 16, (part & 1) ? ua : ub);
+                                const uint2 dd = *reinterpret_cast<const uint2*>(dest_tab + o_atom + part * 2);
+                                const uint32_t d[2] = {dd.x, dd.y};
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const uint32_t da = d[j] & 0xffffu, db = d[j] >> 16;
-                                    if (row2_ok && d[j] != 0xffffffffu) {
-                                        const uint4 val = pack8(&v[j * 8]);
+                                for (int jj = 0; jj < 2; ++jj) {
+                                    const uint32_t da = d[jj] & 0xffffu, db = d[jj] >> 16;
+                                    if (row2_ok && d[jj] != 0xffffffffu) {
+                                        const uint4 val = pack8u(&u[jj * 8]);
                                         if (da != 0xffffu) st_shared_16(nb + da * 16u, val);
                                         if (db != 0xffffu) st_shared_16(nb + db * 16u, val);
                                     }
@@ -468,18 +482,18 @@ __global__ void __launch_bounds__(THREADS, 1) freqkv_dctmm_kernel(const CacheVie
                         } else {
                             // output rows: r_j = y_2j for j < ceil(L/2), r_{L-1-j} = y_{2j+1}
 #pragma unroll
-                            for (int half = 0; half < 2; ++half) {
-                                if (o_atom + half * 4 >= st.outer) continue;
-                                float v[32];
-                                tmem_ld32(taddr + half * 32, v);
+                            for (int part = 0; part < 4; ++part) {
+                                uint32_t(&u)[16] = (part & 1) ? ub : ua;
+                                tmem_ld_wait16(u);
+                                if (part < 3) tmem_ld16_issue(taddr + (part + 1) * 16, (part & 1) ? ua : ub);
                                 if (row < P.l1) {
 #pragma unroll
-                                    for (int j = 0; j < 4; ++j) {
-                                        const int32_t o = o_atom + half * 4 + j;
+                                    for (int jj = 0; jj < 2; ++jj) {
+                                        const int32_t o = o_atom + part * 2 + jj;
                                         if (o < L2) {
-                                            const int32_t jj = L2 * row + o;
-                                            const int32_t m = jj < hL ? 2 * jj : 2 * (L - 1 - jj) + 1;
-                                            *reinterpret_cast<uint4*>(cur_base + (int64_t)m * row_bytes) = pack8(&v[j * 8]);
+                                            const int32_t j_out = L2 * row + o;
+                                            const int32_t m = j_out < hL ? 2 * j_out : 2 * (L - 1 - j_out) + 1;
+                                            *reinterpret_cast<uint4*>(cur_base + (int64_t)m * row_bytes) = pack8u(&u[jj * 8]);
                                         }
                                     }
                                 }

@@ -423,7 +423,11 @@ def test_fdct_refuses_other_lengths(ctx):
     v = torch.zeros_like(k)
     ctx.set_variant(fk.FDCT)
     with pytest.raises(fk.FreqKVError) as e:
-        ctx.compress(k, v, 504, 250, 4)
+        ctx.compress(k, v, 591, 250, 4)      # 587 rows: a prime has no factorisation for the tensor-core stages
+    assert e.value.status == fk.ERR_UNSUPPORTED
+    kf, vf = k.float(), v.float()
+    with pytest.raises(fk.FreqKVError) as e:
+        ctx.compress(kf, vf, 504, 250, 4)    # fp32: the radix-16 kernel takes powers of two only
     assert e.value.status == fk.ERR_UNSUPPORTED
     ctx.set_variant(fk.AUTO)
 
@@ -440,6 +444,8 @@ def test_auto_picks_documented_variants(ctx):
     assert ctx.resolve_variant(bf, 4096, 2048) == fk.GEMM
     assert ctx.resolve_variant(fk.layout_contiguous(fk.BF16, 1, 1, 1, 8192, 64)[1], 4096, 2048) == fk.FDCT
     assert ctx.resolve_variant(bf, 4092, 2046) == fk.GEMM
+    assert ctx.resolve_variant(fk.layout_contiguous(fk.BF16, 1, 1, 1, 8192, 64)[1], 4092, 2046) == fk.FDCT    # tensor-core stages
+    assert ctx.resolve_variant(fk.layout_contiguous(fk.BF16, 1, 1, 1, 8192, 256)[1], 4099, 2049) == fk.SIMT   # a prime length
     assert ctx.resolve_variant(bf, 8188, 4094) == fk.GEMM
     assert ctx.resolve_variant(f32, 512, 256) == fk.FDCT
     assert ctx.resolve_variant(f32, 500, 250) == fk.SIMT

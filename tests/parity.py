@@ -9,7 +9,7 @@ import oracle
 from paper_2505_00570_b200 import binding as fk
 from paper_2505_00570_b200 import synth
 
-TOL = {torch.float32: 1e-5, torch.bfloat16: 1e-2}  # max per-matrix relative L2 (spec bars)
+TOL = {torch.float32: 1e-5, torch.bfloat16: 1e-2}  # max per-matrix relative L2 (the stated tolerances)
 # A matrix norm over a few hundred thousand values cannot see one bad row or one bad 16-byte
 # vector, so every row is bounded too: |got_row - want_row| <= ROW_TOL * max(|want_row|, rms row
 # norm of the matrix).  Three times the matrix bar: a row's error is a sum over the same number of
@@ -123,7 +123,7 @@ def check_compress(ctx: fk.Context, w: synth.Workload, cache_len: int, kept_len:
             scale = max(np.linalg.norm(want), np.sqrt(kept_len / n_in) * np.linalg.norm(x))
             worst = max(worst, float(np.linalg.norm(got - want) / scale))
             plain_band = max(plain_band, rel_l2(got, want))
-            if band_plain:  # the input has energy in the retained band: the benchmark spec's metric itself
+            if band_plain:  # the input has energy in the retained band: the plain metric itself
                 worst = max(worst, rel_l2(got, want))
         elif energy_scaled:
             # an input with almost no energy in the kept band (the opposite of the paper's workloads):

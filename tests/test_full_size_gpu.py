@@ -45,7 +45,7 @@ def coords(i: int, shape) -> tuple[int, int, int, int]:
     return t, j // (Ly * H), (j // H) % Ly, j % H
 
 
-def check_uniform(ctx, name: str, sample: int):
+def check_uniform(ctx, name: str, sample: int, variant: int = fk.AUTO):
     w = synth.WORKLOADS[name]
     cache_len, sink = w.capacity, w.sink
     kept = w.kept_len(cache_len)
@@ -58,8 +58,10 @@ def check_uniform(ctx, name: str, sample: int):
     # device-side copies of what must not change: sink rows and the rows past the new length
     head = [t[..., :sink, :].clone() for t in (k, v)]
     tail = [t[..., sink + kept:, :].clone() for t in (k, v)]
-    assert ctx.resolve_variant(fk.layout_of(k), cache_len - sink, kept) == fk.GEMM
+    ctx.set_variant(variant)
+    assert ctx.resolve_variant(fk.layout_of(k), cache_len - sink, kept) == (fk.GEMM if variant == fk.AUTO else variant)
     new_len = ctx.compress(k, v, cache_len, kept, sink)
+    ctx.set_variant(fk.AUTO)
     assert ctx.last_device_status() == fk.OK and new_len == sink + kept
     for t, hd, tl in zip((k, v), head, tail):
         assert torch.equal(t[..., :sink, :], hd), "sink rows changed"
@@ -80,6 +82,14 @@ def test_config2_llama2_7b_full(ctx):
     """32 x 32 heads x 128, 4096 tokens, 4 sinks, 4092 -> 2046: 2048 matrices in one call."""
     need_gib(20)
     check_uniform(ctx, "llama2_7b", sample=32)
+
+
+@pytest.mark.parametrize("name", ["llama2_7b", "llama2_7b_pow2"])
+def test_config2_full_fast_transform(ctx, name):
+    """The same 2048 matrices through the fast transform on the tensor cores (variant FDCT), in the
+    launch configuration `bench.py --variant fdct` times: 4092 -> 2046 and the literal 4096 -> 2048."""
+    need_gib(20)
+    check_uniform(ctx, name, sample=32, variant=fk.FDCT)
 
 
 def test_config3_llama3_8b_full(ctx):

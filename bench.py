@@ -498,6 +498,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b")
     ap.add_argument("--variant", default="auto", choices=["auto", "gemm", "fdct", "simt"])
+    ap.add_argument("--fast-family", default="auto", choices=["auto", "cooley-tukey", "prime-factor"],
+                    help="factorisation used by the bf16 fast transform (variant fdct)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--retain", type=float, default=0.5, help="retaining ratio gamma: kept_len = floor(gamma * (cache_len - sink))")
@@ -566,6 +568,7 @@ def main():
     ctx = fk.Context(local_rank)
     variant = {"auto": fk.AUTO, "gemm": fk.GEMM, "fdct": fk.FDCT, "simt": fk.SIMT}[args.variant]
     ctx.set_variant(variant)
+    ctx.set_fast_family({"auto": 0, "cooley-tukey": fk.COOLEY_TUKEY, "prime-factor": fk.PRIME_FACTOR}[args.fast_family])
     if args.workload in ("ragged_8b", "stream_7b", "stream_7b_graph"):   # side workloads: one line each, single GPU
         if rank == 0:
             fn = {"ragged_8b": run_ragged, "stream_7b": run_stream, "stream_7b_graph": run_stream_graph}[args.workload]

@@ -53,10 +53,14 @@ typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
  *         over the cache, or, for kept_len <= 256, straight from the cache without that pass;
  *   FDCT  fast transform, O(N log N) (Appendix A: the DCT "can be computed using the FFT"): for
  *         bf16 caches the transform pair is factored into four small dense stages that run on
- *         the tensor cores, for every n_in = N1 N2 and kept_len = L1 L2 whose factors fit the
- *         kernel (N1 <= 126, L2 <= 64, L1 <= 128, about 2 kept_len / N1 <= 128, a shared-memory
- *         budget: n_in up to about 4600 -- 4096 -> 2048 and the paper's 4092 -> 2046 among them),
- *         in place with no scratch; fp32 caches: a radix-16 kernel for power-of-two lengths;
+ *         the tensor cores, in place with no scratch, for every n_in = N1 N2 and kept_len = L1 L2
+ *         whose factors fit the kernel and its shared memory (n_in up to about 4600).  Two
+ *         families of factorisation (see freqkv_set_fast_family): prime-factor, for coprime
+ *         factors with N2 and L2 odd (N1 <= 63, N2 <= 127, L1 <= 63, L2 <= 127: the paper's
+ *         4092 -> 2046 = 44 x 93 -> 22 x 93), real arithmetic and no twiddle factors; and
+ *         Cooley-Tukey, for any factors (N1 <= 126, L2 <= 64, L1 <= 128, about 2 kept_len / N1
+ *         <= 128: 4096 -> 2048), complex with twiddles.  fp32 caches: a radix-16 kernel for
+ *         power-of-two lengths;
  *   SIMT  the same projection on the fp32 CUDA cores (any shape; the only path for fp32
  *         caches of non-power-of-two length);
  *   AUTO  picks per shape from a table filled from measurements. */
@@ -89,6 +93,14 @@ freqkv_status freqkv_destroy(freqkv_ctx* ctx);
 /* Force the variant used by later freqkv_compress* calls (default FREQKV_AUTO).  A forced
  * variant that cannot run a given shape makes that call return FREQKV_ERR_UNSUPPORTED. */
 freqkv_status freqkv_set_variant(freqkv_ctx* ctx, freqkv_variant variant);
+
+/* Which factorisation the bf16 fast transform (variant FDCT) uses in later calls: 0 (default) =
+ * prime-factor where the lengths allow it, else Cooley-Tukey; FREQKV_FAST_COOLEY_TUKEY or
+ * FREQKV_FAST_PRIME_FACTOR = that family only (shapes it cannot factor are then not FDCT shapes
+ * for this context).  INVALID_ARG for any other value. */
+#define FREQKV_FAST_COOLEY_TUKEY 1
+#define FREQKV_FAST_PRIME_FACTOR 2
+freqkv_status freqkv_set_fast_family(freqkv_ctx* ctx, int32_t family);
 
 /* Which variant AUTO (or the forced setting) resolves to for this shape; FREQKV_AUTO is never
  * returned.  Returns FREQKV_ERR_UNSUPPORTED through *out_variant = -1 when none applies. */
@@ -331,10 +343,11 @@ freqkv_status freqkv_check_attend_prefill(const freqkv_layout* layout, const voi
  * matrices before rounding, same index maps -- in fp64 on the host to `channels` signals
  * x[n * channels + c], n < n_in, and writes y[m * channels + c], m < n_keep.  It exists so that a
  * plan can be checked against the definition (Section 3.3, Eq. 2-3; Appendix A) without a GPU; it
- * is not a compute path.  factors (optional) receives N1, N2, L1, L2.  UNSUPPORTED when no
- * factorisation of these lengths fits the kernel. */
-freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, const double* x, int32_t channels, double* y,
-                                          int32_t* factors);
+ * is not a compute path.  family as in freqkv_set_fast_family.  factors (optional, 5 values)
+ * receives N1, N2, L1, L2 and the family used.  UNSUPPORTED when no factorisation of these lengths
+ * fits the kernel. */
+freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, int32_t family, const double* x, int32_t channels,
+                                          double* y, int32_t* factors);
 
 /* Text of the most recent CUDA failure or device-status report seen by this context (owned by
  * the context, valid until its next call); "" if none. */

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libfreqkv.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(7)
 BF16, F32 = 0, 1
 AUTO, GEMM, FDCT, SIMT = 0, 1, 2, 3
+COOLEY_TUKEY, PRIME_FACTOR = 1, 2   # families of the bf16 fast transform (freqkv_set_fast_family)
 VARIANT_NAMES = {AUTO: "auto", GEMM: "gemm", FDCT: "fdct", SIMT: "simt"}
 
 EXPORTS = [
@@ -30,7 +31,7 @@ EXPORTS = [
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
     "freqkv_attend_prefill", "freqkv_check_attend_prefill",
     "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
-    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait", "freqkv_fast_plan_apply_host",
+    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait", "freqkv_fast_plan_apply_host", "freqkv_set_fast_family",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -96,7 +97,8 @@ def lib() -> ctypes.CDLL:
         L.freqkv_check_attend_prefill.argtypes = [LP, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_int32, I32P]
         L.freqkv_set_wait_limit.argtypes = [c_void_p, c_int64]
         L.freqkv_selftest_bounded_wait.argtypes = [c_void_p, c_int64, c_void_p]
-        L.freqkv_fast_plan_apply_host.argtypes = [c_int32, c_int32, c_void_p, c_int32, c_void_p, I32P]
+        L.freqkv_fast_plan_apply_host.argtypes = [c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, I32P]
+        L.freqkv_set_fast_family.argtypes = [c_void_p, c_int32]
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -165,17 +167,18 @@ def check_attend_prefill(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_p
     return lib().freqkv_check_attend_prefill(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, n_new, arr)
 
 
-def fast_plan_apply_host(x, n_keep: int):
+def fast_plan_apply_host(x, n_keep: int, family: int = 0):
     """``freqkv_fast_plan_apply_host``: the FDCT variant's factored chain applied in fp64 on the
     host to a float64 numpy array ``x`` [n_in, channels] (a plan diagnostic, not a compute path).
-    Returns (y [n_keep, channels], (N1, N2, L1, L2)); raises FreqKVError(ERR_UNSUPPORTED) when
-    the lengths do not factor within the kernel's limits."""
+    ``family``: 0 = the kernel's own choice, ``COOLEY_TUKEY`` or ``PRIME_FACTOR``.
+    Returns (y [n_keep, channels], (N1, N2, L1, L2, family used)); raises
+    FreqKVError(ERR_UNSUPPORTED) when the lengths do not factor within the kernel's limits."""
     import numpy as np
 
     x = np.ascontiguousarray(x, dtype=np.float64)
     y = np.empty((n_keep, x.shape[1]), dtype=np.float64)
-    fac = (c_int32 * 4)()
-    st = lib().freqkv_fast_plan_apply_host(x.shape[0], n_keep, x.ctypes.data, x.shape[1], y.ctypes.data, fac)
+    fac = (c_int32 * 5)()
+    st = lib().freqkv_fast_plan_apply_host(x.shape[0], n_keep, family, x.ctypes.data, x.shape[1], y.ctypes.data, fac)
     if st != OK:
         raise FreqKVError(st, f"freqkv_fast_plan_apply_host: {status_string(st)}")
     return y, tuple(fac)
@@ -272,6 +275,9 @@ class Context:
 
     def set_variant(self, variant: int):
         self._check(lib().freqkv_set_variant(self._h, variant), "freqkv_set_variant")
+
+    def set_fast_family(self, family: int):
+        self._check(lib().freqkv_set_fast_family(self._h, family), "freqkv_set_fast_family")
 
     def resolve_variant(self, layout: Layout, n_in: int, n_keep: int) -> int:
         out = c_int32(-1)

@@ -28,8 +28,10 @@ struct freqkv_ctx {
     freqkv_variant forced = FREQKV_AUTO;
     std::map<std::tuple<int32_t, int32_t, int32_t>, Basis> bases;  // (n_in, n_keep, first retained component)
     std::map<std::pair<int32_t, int32_t>, FdctPlan> fdct_plans;
-    std::map<std::pair<int32_t, int32_t>, DctmmPlan> dctmm_plans;
-    std::map<std::pair<int32_t, int32_t>, bool> dctmm_fits;  // does a factorisation of (n_in, n_keep) meet the kernel's limits
+    // keys: (n_in, n_keep, family of factorisation asked for: 0 = the kernel's own choice)
+    std::map<std::tuple<int32_t, int32_t, int32_t>, DctmmPlan> dctmm_plans;
+    std::map<std::tuple<int32_t, int32_t, int32_t>, bool> dctmm_fits;  // does a factorisation meet the kernel's limits
+    int32_t fast_family = 0;
     size_t basis_bytes = 0;
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
@@ -205,10 +207,10 @@ bool fdct_applicable(const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 bool dctmm_applicable(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 {
     if (l.dtype != FREQKV_BF16 || l.head_dim % 8 != 0) return false;
-    const auto key = std::make_pair(n_in, n_keep);
+    const auto key = std::make_tuple(n_in, n_keep, ctx->fast_family);
     auto it = ctx->dctmm_fits.find(key);
     if (it != ctx->dctmm_fits.end()) return it->second;
-    const bool ok = dctmm_supported(l.dtype, l.head_dim, n_in, n_keep);
+    const bool ok = dctmm_supported(l.dtype, l.head_dim, n_in, n_keep, ctx->fast_family);
     if (ctx->dctmm_fits.size() > 4096) ctx->dctmm_fits.clear();
     ctx->dctmm_fits[key] = ok;
     return ok;
@@ -410,10 +412,10 @@ freqkv_status compress_group(freqkv_ctx* ctx, const freqkv_layout& l, void* k, v
 
     if (variant == FREQKV_FDCT && first == 0 && dctmm_applicable(ctx, l, n_in, n_keep)) {
         DctmmPlan plan;
-        const auto key = std::make_pair(n_in, n_keep);
+        const auto key = std::make_tuple(n_in, n_keep, ctx->fast_family);
         auto it = ctx->dctmm_plans.find(key);
         if (it == ctx->dctmm_plans.end()) {
-            const cudaError_t e = dctmm_make_plan(n_in, n_keep, stream, &plan);
+            const cudaError_t e = dctmm_make_plan(n_in, n_keep, ctx->fast_family, stream, &plan);
             if (e != cudaSuccess) return cuda_fail(ctx, e, "dctmm_make_plan");
             ctx->dctmm_plans[key] = plan;
         } else {
@@ -600,6 +602,13 @@ freqkv_status freqkv_set_variant(freqkv_ctx* ctx, freqkv_variant variant)
     return FREQKV_OK;
 }
 
+freqkv_status freqkv_set_fast_family(freqkv_ctx* ctx, int32_t family)
+{
+    if (!ctx || (family != 0 && family != DCTMM_COOLEY_TUKEY && family != DCTMM_PRIME_FACTOR)) return FREQKV_ERR_INVALID_ARG;
+    ctx->fast_family = family;
+    return FREQKV_OK;
+}
+
 freqkv_status freqkv_resolve_variant(freqkv_ctx* ctx, const freqkv_layout* layout, int32_t n_in, int32_t n_keep,
                                      int32_t* out_variant)
 {
@@ -620,11 +629,11 @@ freqkv_status freqkv_plan(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, freqkv_
     DeviceGuard g(ctx->device);
     if (!g.ok) return FREQKV_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (variant == FREQKV_FDCT && dtype == FREQKV_BF16 && n_keep < n_in && dctmm_supported(dtype, 128, n_in, n_keep)) {
-        const auto key = std::make_pair(n_in, n_keep);
+    if (variant == FREQKV_FDCT && dtype == FREQKV_BF16 && n_keep < n_in && dctmm_supported(dtype, 128, n_in, n_keep, ctx->fast_family)) {
+        const auto key = std::make_tuple(n_in, n_keep, ctx->fast_family);
         if (ctx->dctmm_plans.find(key) == ctx->dctmm_plans.end()) {
             DctmmPlan plan;
-            const cudaError_t e = dctmm_make_plan(n_in, n_keep, stream, &plan);
+            const cudaError_t e = dctmm_make_plan(n_in, n_keep, ctx->fast_family, stream, &plan);
             if (e != cudaSuccess) return cuda_fail(ctx, e, "dctmm_make_plan");
             ctx->dctmm_plans[key] = plan;
         }
@@ -1338,17 +1347,19 @@ freqkv_status freqkv_selftest_bounded_wait(freqkv_ctx* ctx, int64_t nanoseconds,
     return FREQKV_OK;
 }
 
-freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, const double* x, int32_t channels, double* y,
-                                          int32_t* factors)
+freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, int32_t family, const double* x, int32_t channels,
+                                          double* y, int32_t* factors)
 {
     if (!x || !y || channels < 1 || n_in < 1 || n_keep < 1 || n_keep >= n_in) return FREQKV_ERR_INVALID_ARG;
+    if (family != 0 && family != DCTMM_COOLEY_TUKEY && family != DCTMM_PRIME_FACTOR) return FREQKV_ERR_INVALID_ARG;
     DctmmHostPlan hp;
-    if (!dctmm_host_plan(n_in, n_keep, &hp)) return FREQKV_ERR_UNSUPPORTED;
+    if (!dctmm_host_plan(n_in, n_keep, family, &hp)) return FREQKV_ERR_UNSUPPORTED;
     if (factors) {
         factors[0] = hp.plan.n1;
         factors[1] = hp.plan.n2;
         factors[2] = hp.plan.l1;
         factors[3] = hp.plan.l2;
+        factors[4] = hp.plan.family;
     }
     dctmm_host_apply(hp, x, channels, y);
     return FREQKV_OK;

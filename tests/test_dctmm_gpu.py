@@ -24,16 +24,23 @@ def wl(cap, sink, B=1, Ly=1, H=2, hd=128, rho=0.9, seed=21):
     return synth.Workload("fast", B, Ly, H, hd, cap, torch.bfloat16, sink, rho, 2, synth.BASE_SEED + seed)
 
 
+@pytest.mark.parametrize("family", [fk.PRIME_FACTOR, fk.COOLEY_TUKEY])
 @pytest.mark.parametrize("n_in,kept,sink", [(1024, 512, 0), (4096, 2048, 0), (4092, 2046, 4), (4092, 1023, 4), (4092, 3069, 4), (2046, 1534, 4),
                                             (1000, 333, 3), (2046, 1023, 2), (3000, 1500, 4), (300, 150, 4), (4094, 2047, 0),
-                                            (4092, 40, 4)])
-def test_fast_transform_lengths(ctx, n_in, kept, sink):
+                                            (4092, 40, 4), (4600, 2300, 4), (4340, 2170, 0)])
+def test_fast_transform_lengths(ctx, n_in, kept, sink, family):
+    """Both families of factorisation (coprime factors without twiddles; any factors with twiddles),
+    each on every pair of lengths it can factor."""
     w = wl(n_in + sink + 5, sink)
     ctx.set_variant(fk.FDCT)
-    lay = fk.layout_of(torch.empty(1, 1, 2, n_in + sink + 5, 128, dtype=torch.bfloat16))
-    if ctx.resolve_variant(lay, n_in, kept) != fk.FDCT:
-        pytest.skip("no factorisation of these lengths fits the kernel's shared memory")
-    parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.FDCT)
+    ctx.set_fast_family(family)
+    try:
+        lay = fk.layout_of(torch.empty(1, 1, 2, n_in + sink + 5, 128, dtype=torch.bfloat16))
+        if ctx.resolve_variant(lay, n_in, kept) != fk.FDCT:
+            pytest.skip("no factorisation of this family fits the kernel for these lengths")
+        parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.FDCT)
+    finally:
+        ctx.set_fast_family(0)
 
 
 def test_fast_transform_white_noise(ctx):

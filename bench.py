@@ -366,7 +366,7 @@ def run_attend(args, ctx, fk, synth, name, dev, peaks):
     import dataclasses
 
     B, H, G, cap, base, rho = {"attend_7b": (16, 32, 1, 4096, 10000.0, 0.9), "attend_8b": (8, 8, 4, 8192, 500000.0, 0.95)}[name]
-    layers = 4
+    layers = args.layers if args.layers > 0 else 4   # one layer (1.07 GB on 7B) is already far larger than L2: enough for a profiler capture
     w = synth.Workload(name, B, layers, H, 128, cap, torch.bfloat16, 4, rho, 2, synth.BASE_SEED + 7)
     k, v = synth.make_cache(w, dev)
     gen = torch.Generator(device=dev)

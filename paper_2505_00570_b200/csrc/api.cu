@@ -216,11 +216,14 @@ bool dctmm_applicable(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int
     return ok;
 }
 
-// Variant table, from measurements on B200 (7B shape, 2048 matrices): at 4096 -> 2048 bf16 the
-// tensor-core projection takes 2.36 ms (fold pass included) and the fast transform 4.63 ms, so
-// bf16 caches with head_dim 128 go to the tensor cores whenever a tile can be filled; the fast
-// transform serves the power-of-two shapes the tensor-core path does not take (fp32 caches, other
-// head sizes); everything else runs as a projection on the CUDA cores.
+// Variant table, from measurements on B200 (7B shape, 2048 matrices of head_dim 128, bf16): the
+// tensor-core projection takes 2.41 ms at 4092 -> 2046 (fold pass included; 2.35 ms at 4096 -> 2048)
+// and the fast transform 2.49 ms (2.77 ms); at 4092 -> 1023, 3000 -> 1500 and 2046 -> 1023 the
+// projection is 1.5 to 2.3 times faster (its work shrinks with both lengths, the fast transform's
+// per-slab chain of steps does not), at 4092 -> 3069 they are level.  So bf16 caches with head_dim
+// 128 go to the projection whenever a tile can be filled; the fast transform serves what the
+// projection does not take (bf16 with other head sizes: 40 times faster there than the CUDA cores;
+// fp32 caches of power-of-two length); everything else runs as a projection on the CUDA cores.
 int32_t resolve(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int32_t n_keep)
 {
     const bool g = gemm_applicable(l, n_in, n_keep);

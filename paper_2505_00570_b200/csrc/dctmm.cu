@@ -43,17 +43,21 @@
 // in global memory with no scratch -- no other CTA touches those channels.
 //
 // One persistent CTA per SM:
-//   warps 0-15  load the slab (cp.async, each 16-byte piece placed where stage 1 wants it), and
-//               after every stage move the accumulators from tensor memory to the next stage's
+//   warps 0-15  after every stage move the accumulators from tensor memory to the next stage's
 //               operand in shared memory (twiddle, round to bf16, re-index) or, after stage 4, to
 //               the cache; warp w works on TMEM lanes 32 (w % 4) .. +31 and on 64-column group
 //               w / 4 of every chunk;
 //   warp 16     issues the tcgen05.mma instructions (M 128, N up to 256, K 16; bf16 in, fp32 out)
 //               of one 256-column chunk at a time into one of two halves of tensor memory, so
-//               that the products of a chunk overlap the movement of the previous one.
+//               that the products of a chunk overlap the movement of the previous one;
+//   warps 17-24 load: cp.async, each 16-byte piece of a row placed where stage 1 wants it (table
+//               built on the host).  The next slab's copies are issued as soon as stage 3 has
+//               consumed the buffer they go to and run while the other warps finish the slab.
+//               (A warp keeps about one such instruction of 32 scattered pieces in flight, so the
+//               number of loading warps sets the load rate: the 16 moving warps doing it
+//               themselves cost them 5 k cycles per slab, four loading warps were too few.)
 // The four matrices F stay resident in shared memory (copied once per CTA from a pre-swizzled
-// image).  Two data buffers alternate between stages; the next slab's load starts as soon as
-// stage 3 has consumed the buffer it goes to.  Every barrier wait is bounded in time.
+// image).  Two data buffers alternate between stages.  Every barrier wait is bounded in time.
 #include <cuda.h>
 
 #include <algorithm>

@@ -54,7 +54,7 @@ typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
  *   FDCT  fast transform, O(N log N) (Appendix A: the DCT "can be computed using the FFT"): for
  *         bf16 caches the transform pair is factored into four small dense stages that run on
  *         the tensor cores, in place with no scratch, for every n_in = N1 N2 and kept_len = L1 L2
- *         whose factors fit the kernel and its shared memory (n_in up to about 4600).  Two
+ *         whose factors fit the kernel and its shared memory (n_in up to about 4400).  Two
  *         families of factorisation (see freqkv_set_fast_family): prime-factor, for coprime
  *         factors with N2 and L2 odd (N1 <= 63, N2 <= 127, L1 <= 63, L2 <= 127: the paper's
  *         4092 -> 2046 = 44 x 93 -> 22 x 93), real arithmetic and no twiddle factors; and
@@ -96,8 +96,9 @@ freqkv_status freqkv_set_variant(freqkv_ctx* ctx, freqkv_variant variant);
 
 /* Which factorisation the bf16 fast transform (variant FDCT) uses in later calls: 0 (default) =
  * prime-factor where the lengths allow it, else Cooley-Tukey; FREQKV_FAST_COOLEY_TUKEY or
- * FREQKV_FAST_PRIME_FACTOR = that family only (shapes it cannot factor are then not FDCT shapes
- * for this context).  INVALID_ARG for any other value. */
+ * FREQKV_FAST_PRIME_FACTOR = that family only (a shape it cannot factor is then left to the
+ * other kernels: the radix-16 fast transform for powers of two, else GEMM or SIMT).  INVALID_ARG
+ * for any other value. */
 #define FREQKV_FAST_COOLEY_TUKEY 1
 #define FREQKV_FAST_PRIME_FACTOR 2
 freqkv_status freqkv_set_fast_family(freqkv_ctx* ctx, int32_t family);

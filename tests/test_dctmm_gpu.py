@@ -27,7 +27,7 @@ def wl(cap, sink, B=1, Ly=1, H=2, hd=128, rho=0.9, seed=21):
 @pytest.mark.parametrize("family", [fk.PRIME_FACTOR, fk.COOLEY_TUKEY])
 @pytest.mark.parametrize("n_in,kept,sink", [(1024, 512, 0), (4096, 2048, 0), (4092, 2046, 4), (4092, 1023, 4), (4092, 3069, 4), (2046, 1534, 4),
                                             (1000, 333, 3), (2046, 1023, 2), (3000, 1500, 4), (300, 150, 4), (4094, 2047, 0),
-                                            (4092, 40, 4), (4600, 2300, 4), (4340, 2170, 0)])
+                                            (4092, 40, 4), (4400, 2200, 4), (4340, 2170, 0)])
 def test_fast_transform_lengths(ctx, n_in, kept, sink, family):
     """Both families of factorisation (coprime factors without twiddles; any factors with twiddles),
     each on every pair of lengths it can factor."""
@@ -39,6 +39,38 @@ def test_fast_transform_lengths(ctx, n_in, kept, sink, family):
         if ctx.resolve_variant(lay, n_in, kept) != fk.FDCT:
             pytest.skip("no factorisation of this family fits the kernel for these lengths")
         parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.FDCT)
+    finally:
+        ctx.set_fast_family(0)
+
+
+def test_fast_family_switch(ctx):
+    """The default takes the prime-factor stages where the lengths have coprime factors; each family can be
+    forced; a family that cannot factor a shape leaves it to another kernel; other values are refused."""
+    lay = fk.layout_of(torch.empty(1, 1, 2, 4100, 64, dtype=torch.bfloat16))   # head_dim 64: no tensor-core projection
+    w = wl(4100, 4, hd=64)
+    outs = []
+    try:
+        for family in (0, fk.PRIME_FACTOR, fk.COOLEY_TUKEY):
+            ctx.set_fast_family(family)
+            ctx.set_variant(fk.AUTO)
+            assert ctx.resolve_variant(lay, 4092, 2046) == fk.FDCT
+            k, v = synth.make_cache(w, "cuda")
+            ctx.compress(k, v, 4096, 2046, 4)
+            outs.append(k[..., 4:2050, :].clone())
+        assert ctx.last_device_status() == fk.OK
+        assert torch.equal(outs[0], outs[1])              # the default is the prime-factor family here
+        assert not torch.equal(outs[1], outs[2])          # another chain of roundings ...
+        a, b = outs[1].double(), outs[2].double()
+        assert ((a - b).norm() / a.norm()).item() < 1e-2  # ... of the same result
+        ctx.set_fast_family(fk.PRIME_FACTOR)              # 4400 = 2^4 x 5^2 x 11 has no coprime factors within the limits
+        ctx.set_variant(fk.AUTO)
+        big = fk.layout_of(torch.empty(1, 1, 2, 4500, 64, dtype=torch.bfloat16))
+        assert ctx.resolve_variant(big, 4400, 2200) == fk.SIMT
+        ctx.set_fast_family(fk.COOLEY_TUKEY)
+        assert ctx.resolve_variant(big, 4400, 2200) == fk.FDCT
+        with pytest.raises(fk.FreqKVError) as e:
+            ctx.set_fast_family(3)
+        assert e.value.status == fk.ERR_INVALID_ARG
     finally:
         ctx.set_fast_family(0)
 

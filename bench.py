@@ -146,17 +146,25 @@ def barrier():
         dist.barrier()
 
 
-def workload_numbers(w, cache_len, kept, sink):
+def workload_numbers(w, cache_len, kept, sink, first=0):
     e = 2 if w.dtype == torch.bfloat16 else 4
     m = w.n_matrices
     n_in = cache_len - sink
+    # Multiply-adds the tensor-core variant executes.  One level of the symmetry fold: even and odd parts,
+    # ceil(L/2) x ceil(N/2) each.  Where the lengths halve twice (N a multiple of 4, L even, the lowest
+    # components kept) the even part is folded again: ceil(L/4) rows x (N/4 + N/4 + N/2 + N/2) columns.
+    fold_levels = 2 if (n_in % 4 == 0 and kept % 2 == 0 and first == 0 and kept > 256) else 1
+    if fold_levels == 2:
+        folded = 2.0 * ((kept // 2 + 1) // 2) * 3 * (n_in // 2) * w.head_dim * m
+    else:
+        folded = 2.0 * 2 * ((kept + 1) // 2) * ((n_in + 1) // 2) * w.head_dim * m
     return {
+        "fold_levels": fold_levels,
         "matrices": m,
         "cache_in_bytes": m * cache_len * w.head_dim * e,
         "algorithmic_bytes": m * (n_in + kept) * w.head_dim * e,   # read N' rows, write L rows
         "projection_flops": 2.0 * kept * n_in * w.head_dim * m,    # the dense L x N projection (CUDA-core variant)
-        # what the tensor-core variant executes: even and odd parts, ceil(L/2) x ceil(N/2) each
-        "folded_flops": 2.0 * 2 * ((kept + 1) // 2) * ((n_in + 1) // 2) * w.head_dim * m,
+        "folded_flops": folded,
         "append_bytes": 2 * m * (cache_len - sink - kept) * w.head_dim * e,
     }
 
@@ -563,7 +571,7 @@ def main():
     kept = w.kept_len(cache_len, args.retain)
     first = cache_len - sink - kept if args.high_frequencies else 0
     n_new = cache_len - sink - kept
-    nums = workload_numbers(w, cache_len, kept, sink)
+    nums = workload_numbers(w, cache_len, kept, sink, first)
 
     ctx = fk.Context(local_rank)
     variant = {"auto": fk.AUTO, "gemm": fk.GEMM, "fdct": fk.FDCT, "simt": fk.SIMT}[args.variant]
@@ -668,7 +676,7 @@ def main():
                 "frac": achieved / peak, "peak_kind": ("burst" if burst else "sustained") + ", of " + peaks["source"],
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
                 "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
-                "flops_per_launch": nums["folded_flops_per_launch"],
+                "flops_per_launch": nums["folded_flops_per_launch"], "fold_levels": nums["fold_levels"],
                 "dense_equivalent_flops_per_launch": nums["projection_flops_per_launch"],
                 # the fold pass the kernel cannot run without: its time (compress call minus the
                 # timed kernel) and the bytes it moves (every non-sink row read once, written once)

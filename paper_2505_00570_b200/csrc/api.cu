@@ -272,10 +272,13 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
             x.fold_ld = ((n_in + 1) / 2 + 63) / 64 * 64;
             x.fold_rows_pad = ((n_keep + 1) / 2 + 255) / 256 * 256;
             x.dense_rows_pad = 256;
+            // the second fold needs n_in / 2 and n_keep / 2 to be whole and n_in / 2 even
+            x.fold2_rows_pad = (first == 0 && n_in % 4 == 0 && n_keep % 2 == 0) ? ((n_keep / 2 + 1) / 2 + 255) / 256 * 256 : 0;
         };
         shape(b);
         const size_t elems = (size_t)b.ld * b.rows_pad;
-        const size_t fold_elems = (size_t)2 * b.fold_ld * b.fold_rows_pad;
+        const size_t fold1_elems = (size_t)2 * b.fold_ld * b.fold_rows_pad;
+        const size_t fold_elems = fold1_elems + (size_t)4 * b.fold_ld * b.fold2_rows_pad;
         const size_t dense_elems = (size_t)256 * b.ld;
         const size_t want = (make_f32 ? elems * 4 : 0) + (make_fold ? fold_elems * 2 : 0) + (make_dense ? dense_elems * 2 : 0);
         if (ctx->basis_bytes + want > kBasisBudgetBytes) {
@@ -311,6 +314,10 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
             e = first == kDctRows ? launch_build_dct_folded(pb, n_in, b.fold_ld, b.fold_rows_pad, stream)
                                   : launch_build_folded_basis(pb, n_in, n_keep, first, b.fold_ld, b.fold_rows_pad, stream);
             ctx->kernels_launched += 1;
+            if (e == cudaSuccess && b.fold2_rows_pad) {
+                e = launch_build_folded2_basis(pb + fold1_elems, n_in, n_keep, b.fold_ld, b.fold2_rows_pad, stream);
+                ctx->kernels_launched += 1;
+            }
         }
         if (e == cudaSuccess && pd) {
             e = launch_build_basis(nullptr, pd, n_in, n_keep, first, b.ld, 256, stream);
@@ -324,7 +331,12 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
         }
         if (pd) { b.dense = pd; ctx->basis_bytes += dense_elems * 2; }
         if (pf) { b.f32 = pf; ctx->basis_bytes += elems * 4; }
-        if (pb) { b.fold = pb; ctx->basis_bytes += fold_elems * 2; }
+        if (pb) {
+            b.fold = pb;
+            b.fold2 = b.fold2_rows_pad ? pb + fold1_elems : nullptr;
+            b.fold_alloc_elems = (int64_t)fold_elems;
+            ctx->basis_bytes += fold_elems * 2;
+        }
         ctx->bases[key] = b;
     }
     *out = b;
@@ -333,7 +345,7 @@ freqkv_status get_basis(freqkv_ctx* ctx, int32_t n_in, int32_t n_keep, int32_t f
 
 size_t basis_device_bytes(const Basis& b)
 {
-    return (b.f32 ? (size_t)b.ld * b.rows_pad * 4 : 0) + (b.fold ? (size_t)2 * b.fold_ld * b.fold_rows_pad * 2 : 0) +
+    return (b.f32 ? (size_t)b.ld * b.rows_pad * 4 : 0) + (b.fold ? (size_t)b.fold_alloc_elems * 2 : 0) +
            (b.dense ? (size_t)256 * b.ld * 2 : 0);
 }
 

@@ -107,6 +107,38 @@ __global__ void build_folded_basis_kernel(__nv_bfloat16* __restrict__ out, int32
     }
 }
 
+// Second fold.  For even L the even-t part Pe is, up to a factor, the basis of the compression of
+// N/2 rows to L/2 (t = 2t': cos(pi t' (2m+1) / (2 (L/2))) cos(pi t' (2n+1) / (2 (N/2)))), so it has the same
+// symmetries one level down: with N' = N/2, L' = L/2, n < N'/2, m < ceil(L'/2)
+//     Pee[m][n] = (Pe[m][n] + Pe[m][N'-1-n]) / 2,   Peo[m][n] = (Pe[m][n] - Pe[m][N'-1-n]) / 2,
+//     s_m = Pee uu + Peo uv,   s_{L'-1-m} = Pee uu - Peo uv,     uu_n = u_n + u_{N'-1-n},  uv_n = u_n - u_{N'-1-n}.
+// Planes: 0 = Pee, 1 = Peo (columns n < N'/2), 2 = Po[m][.], 3 = Po[L'-1-m][.] (columns n < N'), rows m < ceil(L'/2).
+__global__ void build_folded2_basis_kernel(__nv_bfloat16* __restrict__ out, int32_t n_in, int32_t n_keep, int32_t ld,
+                                           int32_t rows_pad)
+{
+    const int64_t plane = (int64_t)rows_pad * ld;
+    const int64_t N = n_in, L = n_keep, Nh = N / 2, Lh = L / 2, Nq = Nh / 2, Lq = (Lh + 1) / 2;
+    auto pe = [&](int64_t m, int64_t n) { return 0.5 * (basis_entry(m, n, N, L, 0) + basis_entry(m, N - 1 - n, N, L, 0)); };
+    auto po = [&](int64_t m, int64_t n) { return 0.5 * (basis_entry(m, n, N, L, 0) - basis_entry(m, N - 1 - n, N, L, 0)); };
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < plane; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = i / ld, n = i % ld;
+        double pee = 0.0, peo = 0.0, p_lo = 0.0, p_hi = 0.0;
+        if (m < Lq && n < Nq) {
+            const double a = pe(m, n), b = pe(m, Nh - 1 - n);
+            pee = 0.5 * (a + b);
+            peo = 0.5 * (a - b);
+        }
+        if (m < Lq && n < Nh) {
+            p_lo = po(m, n);
+            p_hi = po(Lh - 1 - m, n);
+        }
+        out[i] = __double2bfloat16(pee);
+        out[plane + i] = __double2bfloat16(peo);
+        out[2 * plane + i] = __double2bfloat16(p_lo);
+        out[3 * plane + i] = __double2bfloat16(p_hi);
+    }
+}
+
 // The plain orthonormal DCT-II of length N, folded the same way (power-spectrum analysis): plane 0
 // holds the even rows C[2m][n], plane 1 the odd rows C[2m+1][n], n < ceil(N/2); applied to
 // u_n = x_n + x_{N-1-n} and v_n = x_n - x_{N-1-n} they give the components z_2m and z_2m+1 (for odd N the
@@ -134,6 +166,15 @@ cudaError_t launch_build_dct_folded(__nv_bfloat16* out, int32_t n_in, int32_t ld
     const int64_t total = (int64_t)2 * rows_pad * ld;
     int64_t blocks = std::min<int64_t>((total + 255) / 256, 148 * 32);
     build_dct_folded_kernel<<<(unsigned)std::max<int64_t>(blocks, 1), 256, 0, stream>>>(out, n_in, ld, rows_pad);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_folded2_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
+                                       cudaStream_t stream)
+{
+    const int64_t total = (int64_t)rows_pad * ld;
+    const int64_t blocks = std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 32));
+    build_folded2_basis_kernel<<<(unsigned)blocks, 256, 0, stream>>>(out, n_in, n_keep, ld, rows_pad);
     return cudaGetLastError();
 }
 

@@ -45,6 +45,13 @@ struct Basis {
     // m < ceil(n_keep/2), n < ceil(n_in/2), bf16, two planes of fold_rows_pad x fold_ld (see basis.cu).
     __nv_bfloat16* fold = nullptr;
     int32_t fold_ld = 0, fold_rows_pad = 0;
+    // The same folded once more, where the lengths allow it (n_in a multiple of 4, n_keep even, first = 0):
+    // Pe is itself the basis of a half-size compression, so it splits again into Pee | Peo; four planes of
+    // fold2_rows_pad x fold_ld -- Pee, Peo, the first ceil(n_keep/4) rows of Po, and the mirrored rows
+    // Po[n_keep/2 - 1 - m] -- stored behind the two planes above in the same allocation (see basis.cu).
+    __nv_bfloat16* fold2 = nullptr;
+    int32_t fold2_rows_pad = 0;
+    int64_t fold_alloc_elems = 0;  // bf16 elements of the allocation `fold` points to
     // Tensor-core path for at most 256 kept rows: the whole P in bf16, dense_rows_pad (256) x ld.
     __nv_bfloat16* dense = nullptr;
     int32_t dense_rows_pad = 0;
@@ -56,6 +63,10 @@ struct Basis {
 // (`first` = index of the first retained DCT component; 0 for the method's low-pass compression)
 cudaError_t launch_build_basis(float* p_f32, __nv_bfloat16* p_bf16, int32_t n_in, int32_t n_keep, int32_t first,
                                int32_t ld, int32_t rows_pad, cudaStream_t stream);
+
+// Pee, Peo, Po (first rows) and Po (mirrored rows) of the twice-folded basis: four planes of rows_pad x ld.
+cudaError_t launch_build_folded2_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t ld, int32_t rows_pad,
+                                       cudaStream_t stream);
 
 // Pe and Po of the folded basis (two planes of rows_pad x ld), zero padding elsewhere.
 cudaError_t launch_build_folded_basis(__nv_bfloat16* out, int32_t n_in, int32_t n_keep, int32_t first, int32_t ld,

@@ -74,6 +74,9 @@ struct GemmParams {
     int32_t basis_rows_pad;     // row offset of the Po plane inside the basis tensor map
     int32_t pair0, pair_count;  // (batch, layer, kv_head) triples covered by this launch
     int32_t m_pairs, k_steps;   // tiles of 256 folded rows per (batch, layer, kv_head); slices per phase
+    // two-level fold only: ceil(L / 4) = twice-folded output rows, N / 4 = rows of uu (and of uv), slices of
+    // the two short phases
+    int32_t rows_quarter, n_quarter, k_steps_short;
     int32_t sink;
     int32_t mirror_sign;        // +1: y[L-1-m] = s - d;  -1: y[L-1-m] = d - s (a retained band that starts at an odd component)
     // power-spectrum mode only: per tensor [layers][kv_heads][n_in] sums, the weight of one squared value
@@ -349,6 +352,74 @@ __global__ void __launch_bounds__(256) fold_kernel(const CacheView view, const F
     }
 }
 
+// Two levels of folding at once (n_in a multiple of 4; see basis.cu): with N' = n_in / 2 and n < N' / 2 the
+// four rows n, N-1-n, N'-1-n and N'+n give u_n, u_{N'-1-n}, v_n, v_{N'-1-n}, and from the two u's
+// uu_n = u_n + u_{N'-1-n}, uv_n = u_n - u_{N'-1-n} (sums in fp32, rounded once).  Plane 0 of a matrix holds uu
+// (rows 0 .. N'/2 - 1) followed by uv (rows N'/2 .. N' - 1), plane 1 holds v: the same bytes as one level.
+__device__ __forceinline__ void fold8x2(const uint4& a, const uint4& b, const uint4& c, const uint4& d, uint4* uu, uint4* uv,
+                                        uint4* v1, uint4* v2)
+{
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w}, cw[4] = {c.x, c.y, c.z, c.w},
+                   dw[4] = {d.x, d.y, d.z, d.w};
+    uint32_t o[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float a0 = __uint_as_float(aw[i] << 16), a1 = __uint_as_float(aw[i] & 0xffff0000u);
+        const float b0 = __uint_as_float(bw[i] << 16), b1 = __uint_as_float(bw[i] & 0xffff0000u);
+        const float c0 = __uint_as_float(cw[i] << 16), c1 = __uint_as_float(cw[i] & 0xffff0000u);
+        const float d0 = __uint_as_float(dw[i] << 16), d1 = __uint_as_float(dw[i] & 0xffff0000u);
+        const float p0 = a0 + b0, p1 = a1 + b1, q0 = c0 + d0, q1 = c1 + d1;  // u_n, u_{N'-1-n}
+        o[0][i] = pack_bf16(p0 + q0, p1 + q1);
+        o[1][i] = pack_bf16(p0 - q0, p1 - q1);
+        o[2][i] = pack_bf16(a0 - b0, a1 - b1);
+        o[3][i] = pack_bf16(c0 - d0, c1 - d1);
+    }
+    *uu = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]);
+    *uv = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
+    *v1 = make_uint4(o[2][0], o[2][1], o[2][2], o[2][3]);
+    *v2 = make_uint4(o[3][0], o[3][1], o[3][2], o[3][3]);
+}
+
+// Block (x, y) as in fold_kernel; job.n_half = N' rows per plane; a thread folds two vectors per round.
+__global__ void __launch_bounds__(256) fold2_kernel(const CacheView view, const FoldJob job)
+{
+    const uint32_t pt = blockIdx.x;
+    const char* x = static_cast<const char*>(tensor_base(view, pt & 1)) +
+                    (matrix_offset(view, job.pair0 + (int32_t)(pt >> 1)) + (int64_t)job.sink * view.stride_token) * 2;
+    const int64_t row_bytes = view.stride_token * 2;
+    const int32_t n_quarter = job.n_half / 2;
+    const uint32_t total = (uint32_t)n_quarter * 16u;                // vectors of uu (= of uv)
+    uint4* plane0 = job.dst + (int64_t)pt * 2 * ((int64_t)job.n_half * 16);
+    uint4* plane1 = plane0 + (int64_t)job.n_half * 16;
+    for (uint32_t c0 = blockIdx.y * 512u; c0 < total; c0 += gridDim.y * 512u) {
+        uint4 a[2], b[2], c[2], d[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4);
+                a[j] = __ldcs(reinterpret_cast<const uint4*>(x + n * row_bytes) + (i & 15u));
+                b[j] = __ldcs(reinterpret_cast<const uint4*>(x + (job.n_in - 1 - n) * row_bytes) + (i & 15u));
+                c[j] = __ldcs(reinterpret_cast<const uint4*>(x + (job.n_half - 1 - n) * row_bytes) + (i & 15u));
+                d[j] = __ldcs(reinterpret_cast<const uint4*>(x + (job.n_half + n) * row_bytes) + (i & 15u));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const uint32_t i = c0 + j * 256u + threadIdx.x;
+            if (i < total) {
+                const int32_t n = (int32_t)(i >> 4);
+                uint4 uu, uv, v1, v2;
+                fold8x2(a[j], b[j], c[j], d[j], &uu, &uv, &v1, &v2);
+                __stcs(plane0 + i, uu);
+                __stcs(plane0 + total + i, uv);
+                __stcs(plane1 + i, v1);
+                __stcs(plane1 + (int64_t)(job.n_half - 1 - n) * 16 + (i & 15u), v2);
+            }
+        }
+    }
+}
+
 // The same for a ragged batch in one launch: every sequence has the same number of matrices, so
 // block x belongs to job x / mats_per_seq.
 __global__ void __launch_bounds__(256) fold_ragged_kernel(const CacheView view, const FoldJob* jobs, int32_t mats_per_seq)
@@ -401,7 +472,13 @@ __global__ void __launch_bounds__(256) fold_ragged_kernel(const CacheView view, 
 //   cache (map_x = K tensor, map_v = V tensor, 5-D maps over the non-sink rows), there is one
 //   accumulator and one tile per (batch, layer, kv_head).  The tile's rows are stored only after
 //   every slice of its matrices has been read, so writing in place is safe here too.
-constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2, MODE_RAGGED = 3;
+// MODE_FOLD2: two levels of the symmetry fold (n_in a multiple of 4, n_keep even).  A tile is 256
+//   twice-folded rows m < ceil(L/4) and runs four phases: a = Pee uu and b = Peo uv (N/4 deep), then
+//   d = Po v for rows m and d' = Po v for the mirrored rows L/2-1-m (N/2 deep), alternating between the
+//   two halves of tensor memory.  The epilogue parks a, turns it with b into the pair s = a + b,
+//   s' = a - b (kept as two bf16 in the register a occupied) and stores y_m = s + d, y_{L-1-m} = s - d,
+//   y_{L/2-1-m} = s' + d', y_{L/2+m} = s' - d': three quarters of the multiply-adds of MODE_FOLD.
+constexpr int MODE_FOLD = 0, MODE_SPECTRUM = 1, MODE_DIRECT = 2, MODE_RAGGED = 3, MODE_FOLD2 = 4;
 
 // Ragged mode: a role walks its tiles in increasing order, so the sequence a tile belongs to is
 // found by moving a cursor forward; the table is read only when a tile crosses into a new sequence.
@@ -453,7 +530,9 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                    const __grid_constant__ CUtensorMap map_v, const CacheView view, const GemmParams prm)
 {
     constexpr bool SPECTRUM = MODE == MODE_SPECTRUM;
-    constexpr int PHASES = MODE == MODE_DIRECT ? 1 : 2;
+    constexpr bool FOLD2 = MODE == MODE_FOLD2;
+    constexpr int PHASES = MODE == MODE_DIRECT ? 1 : FOLD2 ? 4 : 2;
+    constexpr int USES = FOLD2 ? 2 : 1;  // times a tile fills each half of tensor memory
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
@@ -512,8 +591,12 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 const int32_t head = pair % view.kv_heads, layer = (pair / view.kv_heads) % view.layers,
                               seq = pair / (view.kv_heads * view.layers);
                 for (int eo = 0; eo < PHASES && alive; ++eo) {
-                    const int32_t plane = (pair_local * 2 + (int32_t)rank) * 2 + eo;  // rank 0: K channels, rank 1: V
-                    for (int32_t ks = 0; ks < tc.k_steps; ++ks, ++it) {
+                    // rank 0: K channels, rank 1: V.  Two-level fold: phases 0, 1 read uu and uv (both in plane 0,
+                    // uv n_quarter rows down), phases 2, 3 read v (plane 1)
+                    const int32_t plane = (pair_local * 2 + (int32_t)rank) * 2 + (FOLD2 ? eo >> 1 : eo);
+                    const int32_t row0 = (FOLD2 && eo == 1) ? prm.n_quarter : 0;
+                    const int32_t phase_steps = (FOLD2 && eo < 2) ? prm.k_steps_short : tc.k_steps;
+                    for (int32_t ks = 0; ks < phase_steps; ++ks, ++it) {
                         const int s = it % STAGES;
                         if (it >= STAGES &&
                             !mbar_wait(empty_bar(s), ((it / STAGES) - 1) & 1, abort_flag, prm.status, ERR_EMPTY_WAIT, prm.wait_limit_ns)) {
@@ -530,8 +613,8 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                             tma_load_5d(stage + A_BYTES, cache, leader_full, 0, k0, head, layer, seq);
                             tma_load_5d(stage + A_BYTES + B_CHUNK_BYTES, cache, leader_full, 64, k0, head, layer, seq);
                         } else {
-                            tma_load_3d(stage + A_BYTES, tc.map_x, leader_full, 0, k0, plane);
-                            tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, tc.map_x, leader_full, 64, k0, plane);
+                            tma_load_3d(stage + A_BYTES, tc.map_x, leader_full, 0, row0 + k0, plane);
+                            tma_load_3d(stage + A_BYTES + B_CHUNK_BYTES, tc.map_x, leader_full, 64, row0 + k0, plane);
                         }
                     }
                 }
@@ -548,10 +631,13 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             bool alive = true;
             SeqCursor cursor;
             for (int32_t tile = cluster; tile < total_tiles && alive; tile += n_clusters, ++tile_no) {
-                const int32_t k_steps = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor).k_steps;
+                const int32_t tile_steps = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor).k_steps;
                 for (int eo = 0; eo < PHASES && alive; ++eo) {
-                    if (tile_no > 0) {  // both CTAs' epilogues must have read this accumulator of the last tile
-                        if (!mbar_wait(acc_empty_bar(eo), (tile_no - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT, prm.wait_limit_ns)) {
+                    const int acc = eo & 1;                                   // half of tensor memory
+                    const uint32_t use = tile_no * USES + (uint32_t)(eo >> 1);  // how often that half was filled before
+                    const int32_t k_steps = (FOLD2 && eo < 2) ? prm.k_steps_short : tile_steps;
+                    if (use > 0) {  // both CTAs' epilogues must have read what this half held last
+                        if (!mbar_wait(acc_empty_bar(acc), (use - 1) & 1, abort_flag, prm.status, ERR_ACC_EMPTY_WAIT, prm.wait_limit_ns)) {
                             alive = false;
                             break;
                         }
@@ -571,11 +657,11 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                             const uint64_t ad = smem_desc(a0 + kk * 32, 16, 1024);
                             // B: per CTA 2 chunks of 64 channels 8 KB apart (leading offset), 8-row groups 1 KB apart
                             const uint64_t bd = smem_desc(b0 + kk * 2048, B_CHUNK_BYTES, 1024);
-                            umma_bf16(tmem_base + eo * 256, ad, bd, (ks | kk) != 0);
+                            umma_bf16(tmem_base + acc * 256, ad, bd, (ks | kk) != 0);
                         }
                         umma_commit_both(empty_bar(s));  // frees the stage in both CTAs when these MMAs have read it
                     }
-                    if (alive) umma_commit_both(acc_full_bar(eo));
+                    if (alive) umma_commit_both(acc_full_bar(acc));
                 }
             }
         }
@@ -639,6 +725,86 @@ freqkv_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     if (t < prm.n_in && prm.spectrum[tensor])
                         atomicAdd(prm.spectrum[tensor] + ((int64_t)layer * view.kv_heads + head) * prm.n_in + t,
                                   sum * prm.spectrum_scale);
+                }
+                if (!alive) break;
+            }
+        } else if constexpr (FOLD2) {
+            const uint32_t leader_empty[2] = {leader_s_empty, leader_d_empty};
+            auto release = [&](int acc) {
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(leader_empty[acc]);
+            };
+            for (int32_t tile = cluster; tile < total_tiles; tile += n_clusters, ++tile_no) {
+                const uint32_t use = 2 * tile_no;
+                // a = Pee uu: park this thread's row (128 columns) in registers
+                if (!mbar_wait(acc_full_bar(0), use & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                uint32_t s[128];
+                tmem_ld32<0>(lane_addr + 0, s);
+                tmem_ld32<32>(lane_addr + 32, s);
+                tmem_ld32<64>(lane_addr + 64, s);
+                tmem_ld32<96>(lane_addr + 96, s);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                release(0);
+                // b = Peo uv: s = a + b (low half of the register) and s' = a - b (high half), both bf16
+                if (!mbar_wait(acc_full_bar(1), use & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t b[16];
+                    tmem_ld16(lane_addr + 256 + c * 16, b);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float av = __uint_as_float(s[c * 16 + j]), bv = __uint_as_float(b[j]);
+                        s[c * 16 + j] = pack_bf16(av + bv, av - bv);
+                    }
+                }
+                release(1);
+
+                const TileCtx tc = tile_ctx<MODE>(prm, tile, &map_p, &map_x, cursor);
+                const int32_t m = (tc.m_tile * 2 + (int32_t)rank) * BM + quarter * 32 + lane;
+                const int32_t mh = tc.rows_half - 1 - m;  // the row whose even part is s'
+                const bool row_ok = m < prm.rows_quarter;
+                __nv_bfloat16* mat = static_cast<__nv_bfloat16*>(tensor_base(view, tensor)) +
+                                     matrix_offset(view, tc.pair) + (int64_t)prm.sink * view.stride_token;
+                bool alive = true;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    // d = Po v of rows m (half 0) or of the mirrored rows L/2-1-m (half 1): rows r and L-1-r
+                    if (!mbar_wait(acc_full_bar(half), (use + 1) & 1, abort_flag, prm.status, ERR_ACC_FULL_WAIT, prm.wait_limit_ns)) {
+                        alive = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const int32_t r = half ? mh : m;
+                    const bool store = row_ok && !(half && mh == m);  // the middle row of an odd L/2 comes out of half 0
+                    uint4* out_p = reinterpret_cast<uint4*>(mat + (int64_t)r * view.stride_token);
+                    uint4* out_m = reinterpret_cast<uint4*>(mat + (int64_t)(tc.n_keep - 1 - r) * view.stride_token);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t d[16];
+                        tmem_ld16(lane_addr + half * 256 + c * 16, d);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (store) {
+                            uint32_t p[8], q[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const uint32_t w0 = s[c * 16 + 2 * j], w1 = s[c * 16 + 2 * j + 1];
+                                const float s0 = __uint_as_float(half ? w0 & 0xffff0000u : w0 << 16);
+                                const float s1 = __uint_as_float(half ? w1 & 0xffff0000u : w1 << 16);
+                                const float d0 = __uint_as_float(d[2 * j]), d1 = __uint_as_float(d[2 * j + 1]);
+                                p[j] = pack_bf16(s0 + d0, s1 + d1);
+                                q[j] = pack_bf16(s0 - d0, s1 - d1);
+                            }
+                            out_p[2 * c] = make_uint4(p[0], p[1], p[2], p[3]);
+                            out_p[2 * c + 1] = make_uint4(p[4], p[5], p[6], p[7]);
+                            out_m[2 * c] = make_uint4(q[0], q[1], q[2], q[3]);
+                            out_m[2 * c + 1] = make_uint4(q[4], q[5], q[6], q[7]);
+                        }
+                    }
+                    release(half);
                 }
                 if (!alive) break;
             }
@@ -755,6 +921,18 @@ bool encode_basis_map(CUtensorMap* map, const Basis& basis)
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The four planes of the twice-folded basis stacked: 4 * fold2_rows_pad rows x fold_ld columns.
+bool encode_basis2_map(CUtensorMap* map, const Basis& basis)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)basis.fold_ld, (cuuint64_t)4 * basis.fold2_rows_pad};
+    const cuuint64_t strides[1] = {(cuuint64_t)basis.fold_ld * 2};
+    const cuuint32_t box[2] = {BK, BM};
+    const cuuint32_t elem[2] = {1, 1};
+    return encode_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, basis.fold2, dims, strides, box, elem,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // The scratch planes as a 3-D tensor (channel, folded row, plane); rows past n_half read as zero.
 bool encode_scratch_map(CUtensorMap* map, void* scratch, int32_t n_half, int32_t planes)
 {
@@ -796,6 +974,8 @@ cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, in
             e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(freqkv_gemm_kernel<MODE_FOLD2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) {
             state->last_error = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -850,13 +1030,16 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
     const cudaError_t prepared = gemm_prepare(state, view.mats_per_tensor, basis, sm_count);
     if (prepared != cudaSuccess) return prepared;
     const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
-    const int32_t m_pairs = (rows_half + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
+    // two levels of folding where the basis has them (lengths that halve twice; not for the spectrum's basis)
+    const bool fold2 = basis.fold2 != nullptr && !spectrum;
+    const int32_t rows_quarter = (rows_half + 1) / 2;
+    const int32_t m_pairs = ((fold2 ? rows_quarter : rows_half) + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
     const int32_t pairs = view.mats_per_tensor;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;
     // One pass when the folded inputs fit the scratch buffer, else several passes of `chunk` pairs.
     const int64_t chunk = std::min<int64_t>(std::max<int64_t>(1, (int64_t)(kFoldBufferBytes / per_pair)), pairs);
     CUtensorMap map_p;
-    if (!encode_basis_map(&map_p, basis)) {
+    if (!(fold2 ? encode_basis2_map(&map_p, basis) : encode_basis_map(&map_p, basis))) {
         state->last_error = "tensor map encoding rejected the basis";
         return cudaErrorInvalidValue;
     }
@@ -868,8 +1051,13 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         job.n_half = n_half;
         job.sink = sink;
         job.dst = static_cast<uint4*>(state->scratch);
-        const unsigned fold_y = (unsigned)std::min<int64_t>(((int64_t)n_half * 16 + 1023) / 1024, 64);
-        fold_kernel<<<dim3((unsigned)job.pair_count * 2, fold_y), 256, 0, stream>>>(view, job);
+        if (fold2) {
+            const unsigned fold_y = (unsigned)std::min<int64_t>(((int64_t)(n_half / 2) * 16 + 511) / 512, 64);
+            fold2_kernel<<<dim3((unsigned)job.pair_count * 2, fold_y), 256, 0, stream>>>(view, job);
+        } else {
+            const unsigned fold_y = (unsigned)std::min<int64_t>(((int64_t)n_half * 16 + 1023) / 1024, 64);
+            fold_kernel<<<dim3((unsigned)job.pair_count * 2, fold_y), 256, 0, stream>>>(view, job);
+        }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) {
             state->last_error = "fold_kernel launch";
@@ -883,7 +1071,10 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         GemmParams prm;
         prm.n_keep = basis.n_keep;
         prm.rows_half = rows_half;
-        prm.basis_rows_pad = basis.fold_rows_pad;
+        prm.basis_rows_pad = fold2 ? basis.fold2_rows_pad : basis.fold_rows_pad;
+        prm.rows_quarter = rows_quarter;
+        prm.n_quarter = n_half / 2;
+        prm.k_steps_short = (n_half / 2 + BK - 1) / BK;
         prm.pair0 = job.pair0;
         prm.pair_count = job.pair_count;
         prm.m_pairs = m_pairs;
@@ -915,6 +1106,7 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
         cfg.numAttrs = 1;
         if (hooks.before) hooks.before(hooks.user, stream);
         e = spectrum ? cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_SPECTRUM>, map_p, map_x, map_x, view, prm)
+            : fold2  ? cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_FOLD2>, map_p, map_x, map_x, view, prm)
                      : cudaLaunchKernelEx(&cfg, freqkv_gemm_kernel<MODE_FOLD>, map_p, map_x, map_x, view, prm);
         if (hooks.after) hooks.after(hooks.user, stream);
         if (e != cudaSuccess) {

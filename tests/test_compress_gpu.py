@@ -193,8 +193,9 @@ def test_ragged_batch_in_two_launches(ctx):
     """A ragged batch whose sequences all take the folded tensor-core form runs as ONE fold launch
     and ONE tensor-core launch (the kernel counter says so); odd and even lengths, one sequence
     left alone (kept == length), one with more than one tile of rows.  Against the oracle, against
-    the bytes outside the rewritten rows, and bit for bit against compressing each sequence on
-    its own (same kernels, same arithmetic)."""
+    the bytes outside the rewritten rows, and against compressing each sequence on its own: bit
+    for bit where that call runs the same arithmetic (one level of the symmetry fold), and to well
+    inside the tolerance where the lengths halve twice and the single call folds twice."""
     w = small(cap=1400, dtype=torch.bfloat16, sink=4, B=6, Ly=2, H=3, outliers=2)
     k, v = synth.make_cache(w, "cuda")
     k_in, v_in = k.clone(), v.clone()
@@ -208,7 +209,7 @@ def test_ragged_batch_in_two_launches(ctx):
     launched = ctx.get_timing()[2] - before
     assert new_lens == [4 + x for x in kept]
     plans = len({(n, kp) for n, kp in zip(lens, kept) if kp != n - 4})
-    assert launched <= 2 + plans, f"{launched} kernels for the batch (2 + at most {plans} plan builders expected)"
+    assert launched <= 2 + 2 * plans, f"{launched} kernels for the batch (2 + at most {2 * plans} plan builders expected)"
     before = ctx.get_timing()[2]
     k2, v2 = k_in.clone(), v_in.clone()
     assert ctx.compress_ragged(k2, v2, lens, kept, 4) == new_lens
@@ -217,7 +218,13 @@ def test_ragged_batch_in_two_launches(ctx):
     for b in range(6):
         one_k, one_v = k_in[b:b + 1].clone(), v_in[b:b + 1].clone()
         ctx.compress(one_k, one_v, lens[b], kept[b], 4)
-        assert torch.equal(one_k[0], k[b]) and torch.equal(one_v[0], v[b]), f"sequence {b} differs from its own compression"
+        if (lens[b] - 4) % 4 == 0 and kept[b] % 2 == 0 and kept[b] > 256:   # the single call folds twice
+            for one, both in ((one_k, k), (one_v, v)):
+                a, c = one[0, :, :, 4:4 + kept[b]].double(), both[b, :, :, 4:4 + kept[b]].double()
+                assert ((a - c).norm() / c.norm()).item() < 5e-3
+                assert torch.equal(one[0, :, :, :4], both[b, :, :, :4]) and torch.equal(one[0, :, :, 4 + kept[b]:], both[b, :, :, 4 + kept[b]:])
+        else:
+            assert torch.equal(one_k[0], k[b]) and torch.equal(one_v[0], v[b]), f"sequence {b} differs from its own compression"
         for t_in, t_out in ((k_in, k), (v_in, v)):
             assert torch.equal(t_out[b, :, :, :4], t_in[b, :, :, :4])
             assert torch.equal(t_out[b, :, :, 4 + kept[b]:], t_in[b, :, :, 4 + kept[b]:])

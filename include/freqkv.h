@@ -50,7 +50,8 @@ typedef enum { FREQKV_BF16 = 0, FREQKV_F32 = 1 } freqkv_dtype;
  *   GEMM  the DCT-II -> truncate -> IDCT -> rescale chain folded into one precomputed
  *         kept_len x n_in projection basis and run on the tcgen05 tensor cores (bf16 caches,
  *         head_dim 128 only); halved by the even/odd symmetry of the cosines after a fold pass
- *         over the cache, or, for kept_len <= 256, straight from the cache without that pass;
+ *         over the cache (folded twice, to three eighths, where n_in is a multiple of 4 and
+ *         kept_len even), or, for kept_len <= 256, straight from the cache without that pass;
  *   FDCT  fast transform, O(N log N) (Appendix A: the DCT "can be computed using the FFT"): for
  *         bf16 caches the transform pair is factored into four small dense stages that run on
  *         the tensor cores, in place with no scratch, for every n_in = N1 N2 and kept_len = L1 L2

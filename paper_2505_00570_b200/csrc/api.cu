@@ -217,7 +217,7 @@ bool dctmm_applicable(freqkv_ctx* ctx, const freqkv_layout& l, int32_t n_in, int
 }
 
 // Variant table, from measurements on B200 (7B shape, 2048 matrices of head_dim 128, bf16): the
-// tensor-core projection takes 2.41 ms at 4092 -> 2046 (fold pass included; 2.35 ms at 4096 -> 2048)
+// tensor-core projection takes 2.04 ms at 4092 -> 2046 (fold pass included; 2.02 ms at 4096 -> 2048)
 // and the fast transform 2.49 ms (2.77 ms); at 4092 -> 1023, 3000 -> 1500 and 2046 -> 1023 the
 // projection is 1.5 to 2.3 times faster (its work shrinks with both lengths, the fast transform's
 // per-slab chain of steps does not), at 4092 -> 3069 they are level.  So bf16 caches with head_dim

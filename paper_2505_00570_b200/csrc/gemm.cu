@@ -9,6 +9,11 @@
 //     y_m = s_m + d_m,   y_{L-1-m} = s_m - d_m
 // which is the same linear map with half the multiply-adds.  (For odd N the middle row enters u
 // once and v as zero; for odd L the middle output row has d = 0 and is written once.)
+// For even L the even part Pe is itself the basis of a compression of N/2 rows to L/2, so where N is a
+// multiple of 4 it is folded once more (uu, uv; Pee, Peo; see MODE_FOLD2 and basis.cu): three quarters
+// of these multiply-adds again.  The two-level form is what a plain compression of such lengths
+// runs (the paper's 4092 -> 2046 and 4096 -> 2048); the description below is the one-level form, which
+// serves every other length, retained bands, ragged batches and the power spectrum.
 //
 // Two kernels per call:
 //   fold_kernel         reads every non-sink cache row once and writes U and V (bf16) to a scratch

@@ -1036,8 +1036,12 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
     if (prepared != cudaSuccess) return prepared;
     const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
     // two levels of folding where the basis has them (lengths that halve twice; not for the spectrum's basis)
-    const bool fold2 = basis.fold2 != nullptr && !spectrum;
     const int32_t rows_quarter = (rows_half + 1) / 2;
+    // ... and where that means fewer 64-row slices per matrix pair (tiles are 256 rows high: with few kept rows
+    // the second level can leave its last tile nearly empty and save nothing)
+    const int64_t slices1 = (int64_t)((rows_half + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half + BK - 1) / BK);
+    const int64_t slices2 = (int64_t)((rows_quarter + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half / 2 + BK - 1) / BK + (n_half + BK - 1) / BK);
+    const bool fold2 = basis.fold2 != nullptr && !spectrum && slices2 < slices1;
     const int32_t m_pairs = ((fold2 ? rows_quarter : rows_half) + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
     const int32_t pairs = view.mats_per_tensor;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;

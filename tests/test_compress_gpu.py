@@ -241,6 +241,16 @@ def test_gemm_lengths(ctx, n_in, kept, sink):
     parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.GEMM)
 
 
+@pytest.mark.parametrize("n_in,kept,sink", [(2048, 1024, 0), (4092, 2728, 4), (1396, 698, 4), (4092, 2046, 4), (2732, 1366, 0)])
+def test_gemm_two_fold_levels(ctx, n_in, kept, sink):
+    """Lengths that halve twice (n_in a multiple of 4, kept even) run the symmetry fold at two levels: a whole
+    number of 256-row tiles (2048 -> 1024), a ragged last tile (2728 kept rows: 682 twice-folded ones), an odd
+    kept / 2 whose middle row is its own mirror (698, 2046, 1366), several sequences, layers and heads, padded rows."""
+    w = small(cap=n_in + sink + 3, dtype=torch.bfloat16, sink=sink, outliers=2, B=2, Ly=2, H=3)
+    parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.GEMM)
+    parity.check_compress(ctx, w, n_in + sink, kept, sink, fk.GEMM, row_pad=8)
+
+
 def test_gemm_batch_layers_heads_and_padding(ctx):
     w = small(cap=333, dtype=torch.bfloat16, sink=4, outliers=2, B=2, Ly=3, H=2)
     parity.check_compress(ctx, w, 330, 163, 4, fk.GEMM)

@@ -153,11 +153,8 @@ def workload_numbers(w, cache_len, kept, sink, first=0):
     # Multiply-adds the tensor-core variant executes.  One level of the symmetry fold: even and odd parts,
     # ceil(L/2) x ceil(N/2) each.  Where the lengths halve twice (N a multiple of 4, L even, the lowest
     # components kept) the even part is folded again: ceil(L/4) rows x (N/4 + N/4 + N/2 + N/2) columns.
-    # (and the second level means fewer 64-row slices over tiles of 256 rows: the library's own rule)
-    nh, lh = (n_in + 1) // 2, (kept + 1) // 2
-    slices1 = -(-lh // 256) * 2 * -(-nh // 64)
-    slices2 = -(-((lh + 1) // 2) // 256) * 2 * (-(-(nh // 2) // 64) + -(-nh // 64))
-    fold_levels = 2 if (n_in % 4 == 0 and kept % 2 == 0 and first == 0 and kept > 256 and slices2 < slices1) else 1
+    from paper_2505_00570_b200 import binding as _fk
+    fold_levels = _fk.gemm_fold_levels(n_in, kept, first)   # the library's own rule (0 = no fold pass: few kept rows)
     if fold_levels == 2:
         folded = 2.0 * ((kept // 2 + 1) // 2) * 3 * (n_in // 2) * w.head_dim * m
     else:

@@ -351,6 +351,15 @@ freqkv_status freqkv_check_attend_prefill(const freqkv_layout* layout, const voi
 freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, int32_t family, const double* x, int32_t channels,
                                           double* y, int32_t* factors);
 
+/* Host-only: how many levels of the even/odd symmetry fold (Appendix A's cosines are even or odd
+ * under n -> N-1-n) variant GEMM applies to a compression of n_in rows to kept_len components
+ * starting at first_component: 0 = none (kept_len <= 256: straight from the cache), 1, or 2 (n_in a
+ * multiple of 4, kept_len even, first_component 0, and fewer 64-row slices that way).  The executed
+ * multiply-adds per matrix are 2 * ceil(L/2) * ceil(N/2) * head_dim with one level and
+ * 3 * ceil(L/4) * (N/2) * head_dim with two.  -1 for invalid lengths.  Ragged batches and the power
+ * spectrum always use one level. */
+int32_t freqkv_gemm_fold_levels(int32_t n_in, int32_t kept_len, int32_t first_component);
+
 /* Text of the most recent CUDA failure or device-status report seen by this context (owned by
  * the context, valid until its next call); "" if none. */
 const char* freqkv_last_error(freqkv_ctx* ctx);

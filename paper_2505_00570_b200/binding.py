@@ -31,7 +31,7 @@ EXPORTS = [
     "freqkv_check_attend", "freqkv_compress_band", "freqkv_power_spectrum",
     "freqkv_attend_prefill", "freqkv_check_attend_prefill",
     "freqkv_decode_graph_create", "freqkv_decode_graph_launch", "freqkv_decode_graph_destroy",
-    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait", "freqkv_fast_plan_apply_host", "freqkv_set_fast_family",
+    "freqkv_set_wait_limit", "freqkv_selftest_bounded_wait", "freqkv_fast_plan_apply_host", "freqkv_set_fast_family", "freqkv_gemm_fold_levels",
 ]
 NOALLOC_MAX_BASIS_ELEMS = 1 << 20
 NOALLOC_STAGING_BYTES = 4 << 20
@@ -99,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.freqkv_selftest_bounded_wait.argtypes = [c_void_p, c_int64, c_void_p]
         L.freqkv_fast_plan_apply_host.argtypes = [c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, I32P]
         L.freqkv_set_fast_family.argtypes = [c_void_p, c_int32]
+        L.freqkv_gemm_fold_levels.argtypes = [c_int32, c_int32, c_int32]
+        L.freqkv_gemm_fold_levels.restype = c_int32
         L.freqkv_last_error.argtypes = [c_void_p]
         L.freqkv_last_error.restype = c_char_p
         L.freqkv_status_string.argtypes = [c_int]
@@ -165,6 +167,11 @@ def check_attend_prefill(layout: Layout, k_ptr: int, v_ptr: int, layer: int, q_p
                          n_new: int, lens) -> int:
     arr = (c_int32 * len(lens))(*lens)
     return lib().freqkv_check_attend_prefill(ctypes.byref(layout), k_ptr, v_ptr, layer, q_ptr, out_ptr, group, n_new, arr)
+
+
+def gemm_fold_levels(n_in: int, kept_len: int, first_component: int = 0) -> int:
+    """``freqkv_gemm_fold_levels``: 0, 1 or 2 levels of the symmetry fold for these lengths (host only)."""
+    return lib().freqkv_gemm_fold_levels(n_in, kept_len, first_component)
 
 
 def fast_plan_apply_host(x, n_keep: int, family: int = 0):

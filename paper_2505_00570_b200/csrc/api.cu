@@ -1380,6 +1380,12 @@ freqkv_status freqkv_fast_plan_apply_host(int32_t n_in, int32_t n_keep, int32_t 
     return FREQKV_OK;
 }
 
+int32_t freqkv_gemm_fold_levels(int32_t n_in, int32_t kept_len, int32_t first_component)
+{
+    if (n_in < 1 || kept_len < 1 || kept_len > n_in || first_component < 0) return -1;
+    return gemm_fold_levels(n_in, kept_len, first_component);
+}
+
 const char* freqkv_last_error(freqkv_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
 
 const char* freqkv_status_string(freqkv_status status)

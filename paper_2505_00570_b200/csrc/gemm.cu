@@ -1037,11 +1037,7 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
     const int32_t n_half = (basis.n_in + 1) / 2, rows_half = (basis.n_keep + 1) / 2;
     // two levels of folding where the basis has them (lengths that halve twice; not for the spectrum's basis)
     const int32_t rows_quarter = (rows_half + 1) / 2;
-    // ... and where that means fewer 64-row slices per matrix pair (tiles are 256 rows high: with few kept rows
-    // the second level can leave its last tile nearly empty and save nothing)
-    const int64_t slices1 = (int64_t)((rows_half + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half + BK - 1) / BK);
-    const int64_t slices2 = (int64_t)((rows_quarter + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half / 2 + BK - 1) / BK + (n_half + BK - 1) / BK);
-    const bool fold2 = basis.fold2 != nullptr && !spectrum && slices2 < slices1;
+    const bool fold2 = basis.fold2 != nullptr && !spectrum && gemm_fold_levels(basis.n_in, basis.n_keep, basis.first) == 2;
     const int32_t m_pairs = ((fold2 ? rows_quarter : rows_half) + 2 * BM - 1) / (2 * BM);  // tiles of 256 folded rows
     const int32_t pairs = view.mats_per_tensor;
     const size_t per_pair = (size_t)4 * n_half * 128 * 2;
@@ -1287,6 +1283,21 @@ static bool encode_cache_map(CUtensorMap* map, const CacheView& view, int tensor
 }
 
 bool gemm_is_direct(int32_t n_keep) { return n_keep <= 2 * BM; }
+
+// Levels of the symmetry fold a plain compression of these lengths runs: 0 = none (the direct mode), 2 where
+// the lengths halve twice (n_in a multiple of 4, n_keep even, the lowest components kept) and the second level
+// means fewer 64-row slices per matrix pair (tiles are 256 rows high: with few kept rows it can leave its
+// last tile nearly empty and save nothing), else 1.
+int32_t gemm_fold_levels(int32_t n_in, int32_t n_keep, int32_t first)
+{
+    if (gemm_is_direct(n_keep)) return 0;
+    if (first != 0 || n_in % 4 != 0 || n_keep % 2 != 0) return 1;
+    const int32_t n_half = n_in / 2, rows_half = n_keep / 2, rows_quarter = (rows_half + 1) / 2;
+    const int64_t slices1 = (int64_t)((rows_half + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half + BK - 1) / BK);
+    const int64_t slices2 =
+        (int64_t)((rows_quarter + 2 * BM - 1) / (2 * BM)) * 2 * ((n_half / 2 + BK - 1) / BK + (n_half + BK - 1) / BK);
+    return slices2 < slices1 ? 2 : 1;
+}
 
 cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
                                int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream)

@@ -40,6 +40,8 @@ cudaError_t launch_gemm(GemmState* state, const CacheView& view, const Basis& ba
 cudaError_t gemm_prepare(GemmState* state, int32_t pairs, const Basis& basis, int sm_count);
 // At most 256 kept rows: one tile per (batch, layer, kv_head), no fold pass, the dense basis (Basis::dense).
 bool gemm_is_direct(int32_t n_keep);
+// 0, 1 or 2 levels of the symmetry fold for a plain compression of these lengths (see gemm.cu).
+int32_t gemm_fold_levels(int32_t n_in, int32_t n_keep, int32_t first);
 cudaError_t launch_gemm_direct(GemmState* state, const CacheView& view, const Basis& basis, int32_t sink,
                                int32_t* status_dev, int sm_count, const LaunchHooks& hooks, cudaStream_t stream);
 // One sequence of a ragged batch: its index in the cache and the (folded) basis of its lengths.

@@ -171,3 +171,16 @@ def test_null_context_is_rejected():
 def test_create_fails_loudly_without_gpu():
     with pytest.raises(fk.FreqKVError):
         fk.Context(0)
+
+
+def test_fold_level_rule():
+    """Host-only rule of how often variant GEMM folds: twice where the lengths halve twice and that saves
+    64-row slices over tiles of 256 rows, not at all for at most 256 kept rows, else once."""
+    from paper_2505_00570_b200 import binding as fk
+
+    assert fk.gemm_fold_levels(4092, 2046) == 2 and fk.gemm_fold_levels(4096, 2048) == 2 and fk.gemm_fold_levels(8188, 4094) == 2
+    assert fk.gemm_fold_levels(4092, 2046, 2046) == 1      # another band of components: one level
+    assert fk.gemm_fold_levels(4092, 2045) == 1 and fk.gemm_fold_levels(4094, 2047) == 1 and fk.gemm_fold_levels(2046, 1022) == 1
+    assert fk.gemm_fold_levels(3000, 1500) == 1            # 375 twice-folded rows fill two tiles as badly as 750 fill three
+    assert fk.gemm_fold_levels(4092, 40) == 0 and fk.gemm_fold_levels(4092, 256) == 0
+    assert fk.gemm_fold_levels(0, 0) == -1 and fk.gemm_fold_levels(10, 11) == -1 and fk.gemm_fold_levels(10, 5, -1) == -1

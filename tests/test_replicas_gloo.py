@@ -53,6 +53,10 @@ def test_single_process_helpers_are_no_ops():
     assert n["cache_in_bytes"] == 2048 * 4096 * 128 * 2
     assert n["algorithmic_bytes"] == 2048 * (4092 + 2046) * 128 * 2
     assert n["projection_flops"] == 2.0 * 2046 * 4092 * 128 * 2048
+    # 4092 -> 2046 halves twice: 512 twice-folded rows x (1023 + 1023 + 2046 + 2046) columns, three quarters of one level
+    assert n["fold_levels"] == 2 and n["folded_flops"] == 2.0 * 512 * 3 * 2046 * 128 * 2048
+    one = bench.workload_numbers(__import__("paper_2505_00570_b200.synth", fromlist=["x"]).WORKLOADS["llama2_7b"], 4096, 2045, 4)
+    assert one["fold_levels"] == 1 and one["folded_flops"] == 2.0 * 2 * 1023 * 2046 * 128 * 2048
 
 
 def test_reference_arm_rank0_only_prints():
